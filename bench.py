@@ -1,0 +1,483 @@
+#!/usr/bin/env python
+"""Benchmark of libqknorm's hot path: layerwise QK-RMSNorm through the C ABI.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload C5] [--no-table]
+
+One "step" is one pass of the whole hot path (load, per-shard sum of squares,
+combine, gamma multiply, scale, store; Q and K in one launch) over one batch of
+synthetic input of the named workload.  Rank 0 prints ONE JSON line.
+
+ * value        whole-job GB/s (algorithmic bytes: every element read once and
+                written once, every gamma read once), inputs resident in HBM.
+ * e2e          the same metric when every step also copies that step's inputs
+                from pinned host memory and reads the result back.
+ * roofline     the kernel against the measured HBM copy rate of this machine.
+ * cpu_baseline the fp64 CPU oracle, timed on this machine's host cores on a bounded
+                sample of the same workload (a reported baseline, not a target).
+ * configs      the other workloads (us/call, GB/s, fraction of the HBM peak;
+                decode sizes also under CUDA-graph replay).
+
+With N > 1 (torchrun) every rank runs the same workload on its own GPU on its
+own tokens: the path shards by token range with no exchange, so there is no
+collective on the data path ("scaling": "weak").
+
+--impl reference times the CPU oracle as it stands (there is no other
+implementation of the paper to run): rank 0 only, each step a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2608_09160_b200 import workloads as W  # noqa: E402
+
+METRIC = "qknorm_prefill_GBps"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes (read + write) per launch of the dominant kernel measured by ncu
+# (dram__bytes_read.sum + dram__bytes_write.sum); the capture each figure comes
+# from is summarised under profiles/.  None = not captured.
+NCU_DRAM_TRAFFIC_BYTES = {}
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            with open(p) as fh:
+                return float(json.load(fh)["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.samples = []
+        self.proc = None
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.cmd = ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}",
+                        "--format=csv,noheader,nounits", "-lms", "50"]
+        except Exception:
+            self.cmd = None
+
+    def start(self):
+        if self.cmd is None:
+            return
+        try:
+            self.proc = subprocess.Popen(self.cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for s in self.samples:
+            parts = [p.strip() for p in s.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "power_w_max": max(power) if power else None, "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------
+# one workload on one GPU
+# ---------------------------------------------------------------------------------
+class DeviceCase:
+    """Device (and optionally pinned host) buffers of one workload at one shard
+    count, plus the closure that makes the one C-ABI call."""
+
+    def __init__(self, w: W.Workload, S: int, seed_offset: int = 0, host: bool = False):
+        from paper_2608_09160_b200 import binding
+        self.binding = binding
+        self.w, self.S = w, S
+        ww = W.Workload(**{**w.__dict__, "seed": w.seed + seed_offset})
+        inp = W.make_inputs(ww)
+        self.host_in = None
+        if S == 1:
+            host_parts = {"q": [inp["q"]], "k": [inp["k"]], "gq": [inp["gamma_q"]], "gk": [inp["gamma_k"]]}
+        else:
+            host_parts = {"q": W.shard_columns(inp["q"], S), "k": W.shard_columns(inp["k"], S),
+                          "gq": W.shard_columns(inp["gamma_q"], S), "gk": W.shard_columns(inp["gamma_k"], S)}
+        del inp
+        self.dev = {k: [t.cuda() for t in v] for k, v in host_parts.items()}
+        if w.in_place:
+            self.out_q, self.out_k = self.dev["q"], self.dev["k"]
+        else:
+            self.out_q = [torch.empty_like(t) for t in self.dev["q"]]
+            self.out_k = [torch.empty_like(t) for t in self.dev["k"]]
+        if host:
+            self.host_in = {k: [t.pin_memory() for t in host_parts[k]] for k in ("q", "k")}
+            self.host_out = {"q": [torch.empty_like(t).pin_memory() for t in host_parts["q"]],
+                             "k": [torch.empty_like(t).pin_memory() for t in host_parts["k"]]}
+        self.bytes = w.algorithmic_bytes
+
+    def call(self):
+        b, d = self.binding, self.dev
+        if self.S == 1:
+            b.qknorm_fwd(d["q"][0], d["k"][0], d["gq"][0], d["gk"][0], self.w.eps, self.out_q[0], self.out_k[0])
+        else:
+            b.qknorm_fwd_sharded(d["q"], d["k"], d["gq"], d["gk"], self.w.eps, self.out_q, self.out_k)
+
+    def e2e_step(self):
+        """Inputs from pinned host memory, the call, the result back to pinned host memory."""
+        for name in ("q", "k"):
+            for dst, src in zip(self.dev[name], self.host_in[name]):
+                dst.copy_(src, non_blocking=True)
+        self.call()
+        for name, outs in (("q", self.out_q), ("k", self.out_k)):
+            for dst, src in zip(self.host_out[name], outs):
+                dst.copy_(src, non_blocking=True)
+
+    def e2e_bytes(self):
+        n = sum(t.numel() * 2 for name in ("q", "k") for t in self.host_in[name])
+        return n, n
+
+
+def time_calls(fn, steps: int, warmup: int):
+    """Per-call device times (ms) with CUDA events on the current stream."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in evs]
+
+
+def time_region(fn, steps: int):
+    """Total device time (ms) of `steps` back-to-back calls."""
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(steps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b)
+
+
+def graph_replay_us(case: DeviceCase, calls_per_graph: int = 50, replays: int = 20) -> float:
+    """us per call when `calls_per_graph` calls are captured in one CUDA graph and replayed."""
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        for _ in range(3):
+            case.call()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(calls_per_graph):
+            case.call()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(replays):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b) * 1e3 / calls_per_graph)
+    return statistics.median(ts)
+
+
+def config_table(steps: int, warmup: int, peak: float, skip: str):
+    """us/call, GB/s and roofline fraction of every workload other than the headline one."""
+    from paper_2608_09160_b200 import binding
+    rows = {}
+    for name, w in W.WORKLOADS.items():
+        for S in w.shards:
+            key = f"{name}/S{S}"
+            if key == skip:
+                continue
+            case = DeviceCase(w, S)
+            ts = time_calls(case.call, max(steps, 10), max(warmup, 3))
+            med, mn = statistics.median(ts), min(ts)
+            row = {"us_median": round(med * 1e3, 3), "us_min": round(mn * 1e3, 3),
+                   "GBps": round(case.bytes / (med * 1e-3) / 1e9, 1),
+                   "frac_measured_peak": round(case.bytes / (med * 1e-3) / 1e9 / peak, 4),
+                   "frac_nominal_8TBps": round(case.bytes / (med * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
+                   "bytes": case.bytes, "variant": binding.last_variant(),
+                   "l2": "resident (working set < L2)" if case.bytes < 100e6 else "inputs larger than L2"}
+            if w.tokens <= 1024:
+                row["us_graph_replay"] = round(graph_replay_us(case), 3)
+            rows[key] = row
+            del case
+            torch.cuda.empty_cache()
+    return rows
+
+
+# ---------------------------------------------------------------------------------
+# the CPU oracle, timed
+# ---------------------------------------------------------------------------------
+def oracle_sample_inputs(w: W.Workload, tokens: int):
+    import numpy as np  # noqa: F401
+    ws = W.scaled(w, tokens)
+    inp = W.make_inputs(ws)
+    return ws, {k: W.bf16_bits(v) for k, v in inp.items()}
+
+
+def run_oracle_once(bits, eps, nthreads):
+    import oracle
+    t0 = time.perf_counter()
+    oracle.rmsnorm(bits["q"], bits["gamma_q"], eps, nthreads=nthreads)
+    oracle.rmsnorm(bits["k"], bits["gamma_k"], eps, nthreads=nthreads)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(w: W.Workload, target_cpu_seconds: float = 16.0):
+    """Times the oracle on a bounded sample (first `n` tokens' worth of the same
+    recipe) with all host cores; sized so that it costs ~10-30 s of CPU work."""
+    import oracle
+    cores = min(os.cpu_count() or 1, oracle.max_threads())
+    ws, bits = oracle_sample_inputs(w, 256)
+    run_oracle_once(bits, w.eps, cores)                       # warm (builds/loads the library)
+    dt = run_oracle_once(bits, w.eps, cores)
+    cpu_s_per_token = dt * cores / 256
+    n = int(max(256, min(w.tokens, target_cpu_seconds / max(cpu_s_per_token, 1e-9))))
+    ws, bits = oracle_sample_inputs(w, n)
+    dt = run_oracle_once(bits, w.eps, cores)
+    gbs = ws.algorithmic_bytes / dt / 1e9
+    return {"value": round(gbs, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n} of {w.tokens} tokens of {w.name} (dq={w.dq}, dk={w.dk}), "
+                      f"unsharded definition, one pass, {dt:.2f} s wall",
+            "seconds": round(dt, 3)}
+
+
+def run_reference(args):
+    """--impl reference: the oracle as it stands, on host cores, rank 0 only."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    w = W.WORKLOADS[args.workload]
+    cores = min(os.cpu_count() or 1, oracle.max_threads())
+    ws, bits = oracle_sample_inputs(w, 256)
+    run_oracle_once(bits, w.eps, cores)
+    dt = run_oracle_once(bits, w.eps, cores)
+    # each step about 1.5 s of wall time, bounded by the workload itself
+    n = int(max(64, min(w.tokens, 256 * 1.5 / max(dt, 1e-9))))
+    ws, bits = oracle_sample_inputs(w, n)
+    for _ in range(args.warmup):
+        run_oracle_once(bits, w.eps, cores)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run_oracle_once(bits, w.eps, cores)
+    total = time.perf_counter() - t0
+    gbs = ws.algorithmic_bytes * args.steps / total / 1e9
+    sample = f"each step = first {n} of {w.tokens} tokens of {w.name} (dq={w.dq}, dk={w.dk}), fp64 oracle"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": round(gbs, 4), "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(total / args.steps * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "tokens": w.tokens, "dq": w.dq, "dk": w.dk, "sample_tokens": n},
+        "cpu_baseline": {"value": round(gbs, 4), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(gbs, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ---------------------------------------------------------------------------------
+# main
+# ---------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C5", choices=sorted(W.WORKLOADS))
+    ap.add_argument("--shards", type=int, default=0, help="shard count (default: the workload's first)")
+    ap.add_argument("--tokens", type=int, default=0, help="override the token count (for profiling a small case)")
+    ap.add_argument("--no-table", action="store_true", help="skip the per-config table")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        log("note: fewer than 3 warm-up steps requested")
+
+    if args.impl == "reference":
+        return run_reference(args)
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    from paper_2608_09160_b200 import binding, build
+    if rank == 0:
+        build.build()
+    if dist is not None:
+        dist.barrier()
+    binding.load()
+
+    w = W.WORKLOADS[args.workload]
+    if args.tokens:
+        w = W.scaled(w, args.tokens)
+    S = args.shards or w.shards[0]
+    peak, peak_kind = measured_peak()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    case = DeviceCase(w, S, seed_offset=1000 * rank, host=not args.no_e2e)
+
+    # ---- device-resident timing -----------------------------------------------------------
+    for _ in range(args.warmup):
+        case.call()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    n0 = binding.launch_count()
+    barrier()
+    per_call = time_calls(case.call, args.steps, 0)          # one event pair per launch
+    barrier()
+    total_ms = time_region(case.call, args.steps)            # the K timed steps, back to back
+    barrier()
+    launches = binding.launch_count() - n0
+    clocks = sampler.stop()
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * case.bytes / (ms_per_step * 1e-3) / 1e9
+    launch_ms = statistics.mean(per_call)
+    achieved = case.bytes / (launch_ms * 1e-3) / 1e9
+
+    # ---- end to end: host buffers in, host buffers out ----------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        for _ in range(2):
+            case.e2e_step()
+        barrier()
+        e_ms = time_region(case.e2e_step, args.steps)
+        barrier()
+        if dist is not None:
+            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        h2d, d2h = case.e2e_bytes()
+        e2e = {"value": round(world * case.bytes / (e_ms / args.steps * 1e-3) / 1e9, 3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": round(e_ms / args.steps, 3)}
+    variant = binding.last_variant()
+    del case
+    torch.cuda.empty_cache()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    table = None
+    if not args.no_table and world == 1:
+        table = config_table(args.steps, args.warmup, peak, skip=f"{w.name}/S{S}")
+    cpu = None
+    if not args.no_cpu and world == 1:
+        cpu = cpu_baseline(w)
+
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{w.name}: {w.note}", "tokens": w.tokens, "dq": w.dq, "dk": w.dk,
+                   "num_shards": S, "in_place": w.in_place, "storage": "bf16", "eps": w.eps,
+                   "bytes_per_step_per_gpu": w.algorithmic_bytes, "parallelism": f"token-range x{world}, no collective",
+                   "l2": "inputs larger than L2 (no flush needed)" if w.algorithmic_bytes > 300e6
+                         else "working set fits in L2 (L2-warm number)",
+                   "kernel_variant": variant},
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": UNIT,
+                     "frac": round(achieved / peak, 4), "traffic": NCU_DRAM_TRAFFIC_BYTES.get(f"{w.name}/S{S}"),
+                     "peak_kind": f"{peak_kind} copy rate (of {peak_kind})",
+                     "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4),
+                     "algorithmic_bytes_per_launch": w.algorithmic_bytes,
+                     "launch_us_mean": round(launch_ms * 1e3, 3), "launch_us_min": round(min(per_call) * 1e3, 3)},
+        "cpu_baseline": cpu,
+    }
+    if table is not None:
+        line["configs"] = table
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,134 @@
+/*
+ * libqknorm -- layerwise Query-Key RMSNorm for NVIDIA B200 (sm_100a).
+ *
+ * The operation (Eq. 1 of the paper, Section II-A): every token's full
+ * projected Q vector, and separately its full K vector, is replaced by
+ *
+ *     y[j] = x[j] / sqrt( (1/H) * sum_j x[j]^2 + eps ) * gamma[j]
+ *
+ * with H the FULL width of that vector (dq for Q, dk for K), one statistic per
+ * token per tensor ("layerwise": one factor for the whole vector, not one per
+ * head).  The statistic is formed the way Algorithm 1 forms it: a per-shard
+ * partial sum of squares in fp32 (Phase A), the partials combined as scalars in
+ * ascending shard order in fp32 (Phase B, "P2P reduction"),
+ * rstd = 1/sqrt(S_global/H_total + eps), and a single write of
+ * (x * gamma) * rstd (Phases B/C).  On one GPU the shards are logical: separate
+ * device buffers that hold equal contiguous column slices.
+ *
+ * Conventions for every entry point
+ *  - Data pointers are DEVICE pointers.  Activations and gammas are bf16 stored
+ *    as 16-bit words; rows are contiguous (leading dimension = width).
+ *  - Pointer ARRAYS (the *_shards arguments) are HOST arrays of device pointers.
+ *    They are read during the call only and may be freed on return.
+ *  - Ownership: the caller owns every buffer.  The library allocates nothing on
+ *    the device, frees nothing, and keeps no state except a per-device cache of
+ *    the SM count and kernel occupancy.
+ *  - Asynchrony: work is enqueued on `stream` (a cudaStream_t passed as void*;
+ *    NULL = the legacy default stream) and the call returns without
+ *    synchronising.  No cudaMalloc, no cudaMemcpy, no host synchronisation.
+ *  - Errors: the return value is a qknorm_status.  On any error nothing has
+ *    been launched.  tokens == 0 returns QKNORM_OK without a launch.
+ *  - A tensor can be skipped: dq == 0 (with its pointers ignored) means "K
+ *    only", dk == 0 means "Q only".
+ *  - Aliasing: an output may be exactly its own input (in-place, per shard).
+ *    Any other overlap between an output and any other buffer of the call is
+ *    rejected with QKNORM_ERR_ALIAS.
+ *  - Precision: inputs are widened to fp32 (exact), sums of squares and all
+ *    arithmetic are fp32, the product x*gamma*rstd is rounded ONCE to bf16
+ *    (round to nearest even).  Subnormals are kept.  Results are bitwise
+ *    reproducible run to run (no atomics).
+ *  - Fast path: when every base pointer is 16-byte aligned and every (shard)
+ *    width is a multiple of 8 elements, vectorised kernels run; any other
+ *    width or alignment is served by a slower general kernel, not an error.
+ */
+#ifndef QKNORM_H_
+#define QKNORM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QKNORM_MAX_DIM 65536   /* largest dq or dk */
+#define QKNORM_MAX_SHARDS 16   /* largest num_shards */
+
+typedef enum {
+  QKNORM_OK = 0,
+  QKNORM_ERR_NULL = 1,    /* a required pointer is NULL */
+  QKNORM_ERR_SHAPE = 2,   /* tokens < 0, a width < 0 or > QKNORM_MAX_DIM, width not divisible by num_shards, or dq == dk == 0 with tokens > 0 */
+  QKNORM_ERR_ALIGN = 3,   /* a bf16 pointer is not 2-byte aligned, or an fp32 pointer not 4-byte aligned */
+  QKNORM_ERR_ALIAS = 4,   /* an output overlaps another buffer without being exactly its own input */
+  QKNORM_ERR_SHARDS = 5,  /* num_shards < 1 or > QKNORM_MAX_SHARDS */
+  QKNORM_ERR_EPS = 6,     /* eps < 0 or NaN */
+  QKNORM_ERR_CUDA = 7     /* a CUDA call failed; see qknorm_last_cuda_error() */
+} qknorm_status;
+
+/*
+ * qknorm_fwd -- Eq. 1 on unsharded rows (the problem statement of Section II-A;
+ * Algorithm 1 with N = 1).
+ *   q        [tokens, dq] bf16, device, read      k        [tokens, dk] bf16, device, read
+ *   gamma_q  [dq] bf16, device, read              gamma_k  [dk] bf16, device, read
+ *   out_q    [tokens, dq] bf16, device, written   out_k    [tokens, dk] bf16, device, written
+ *   out_q may equal q and out_k may equal k (in place).
+ */
+int qknorm_fwd(const void* q, const void* k, const void* gamma_q, const void* gamma_k,
+               int64_t tokens, int32_t dq, int32_t dk, float eps,
+               void* out_q, void* out_k, void* stream);
+
+/*
+ * qknorm_fwd_sharded -- the same result when each row is held as num_shards
+ * equal column slices in separate buffers (Section III-A, Algorithm 1 Phases
+ * A-C with N = num_shards logical ranks on one GPU).  Slice s holds columns
+ * [s*w, (s+1)*w) of the full row, w = dq/num_shards (resp. dk/num_shards);
+ * gamma is sliced the same way (W_local of Algorithm 1).  dq and dk are the FULL
+ * widths (H_total): the mean is over the whole vector.
+ *   q_shards, k_shards, gamma_q_shards, gamma_k_shards, out_q_shards, out_k_shards:
+ *     HOST arrays of num_shards device pointers; q_shards[s] is [tokens, dq/num_shards], etc.
+ *   out_*_shards[s] may equal the matching input shard (in place).
+ */
+int qknorm_fwd_sharded(const void* const* q_shards, const void* const* k_shards,
+                       const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                       int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
+                       void* const* out_q_shards, void* const* out_k_shards, void* stream);
+
+/*
+ * The *_ex forms run the same kernels and additionally store the statistic, so
+ * that tests can check it on its own (Algorithm 1: S_local, RMS^-1).
+ *   rstd_q, rstd_k         [tokens] fp32, device, written; NULL = not wanted
+ *   partials_q, partials_k [num_shards, tokens] fp32, device, written; NULL = not wanted.
+ *                          partials[s*tokens + t] is shard s's own sum of squares for token t
+ *                          (the scalar each rank would publish in Phase A).
+ */
+int qknorm_fwd_ex(const void* q, const void* k, const void* gamma_q, const void* gamma_k,
+                  int64_t tokens, int32_t dq, int32_t dk, float eps,
+                  void* out_q, void* out_k, float* rstd_q, float* rstd_k, void* stream);
+
+int qknorm_fwd_sharded_ex(const void* const* q_shards, const void* const* k_shards,
+                          const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                          int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
+                          void* const* out_q_shards, void* const* out_k_shards,
+                          float* partials_q, float* partials_k, float* rstd_q, float* rstd_k,
+                          void* stream);
+
+/* Human-readable name of a qknorm_status (static storage, never NULL). */
+const char* qknorm_status_string(int status);
+
+/* The cudaError_t of the last failing CUDA call made by this thread inside the
+ * library (0 if none). */
+int qknorm_last_cuda_error(void);
+
+/* Name of the kernel variant the last successful call on this thread launched
+ * ("rows", "general", "none"); static storage.  For tests and benchmarks. */
+const char* qknorm_last_variant(void);
+
+/* Number of kernel launches this thread has enqueued through the library. */
+int64_t qknorm_launch_count(void);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int qknorm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QKNORM_H_ */

@@ -1,0 +1,221 @@
+"""Thin Python binding of libqknorm's C ABI (argument marshalling only).
+
+Every function here has the name and the arguments of the C entry point it
+calls (see include/qknorm.h).  Tensors are used for their device pointers and
+shapes; all arithmetic happens in the CUDA kernels.  There is no fallback: if
+the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libqknorm.so")
+
+EXPORTS = (
+    "qknorm_fwd",
+    "qknorm_fwd_sharded",
+    "qknorm_fwd_ex",
+    "qknorm_fwd_sharded_ex",
+    "qknorm_status_string",
+    "qknorm_last_cuda_error",
+    "qknorm_last_variant",
+    "qknorm_launch_count",
+    "qknorm_version",
+)
+
+QKNORM_OK = 0
+QKNORM_ERR_NULL = 1
+QKNORM_ERR_SHAPE = 2
+QKNORM_ERR_ALIGN = 3
+QKNORM_ERR_ALIAS = 4
+QKNORM_ERR_SHARDS = 5
+QKNORM_ERR_EPS = 6
+QKNORM_ERR_CUDA = 7
+
+
+class QKNormError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(message)
+        self.status = status
+
+
+_lib = None
+_vp = ctypes.c_void_p
+_vpp = ctypes.POINTER(ctypes.c_void_p)
+
+
+def load() -> ctypes.CDLL:
+    """Loads libqknorm.so (built by ``python -m paper_2608_09160_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise QKNormError(-1, f"{LIB_PATH} is missing: build it with "
+                              f"`python -m paper_2608_09160_b200.build` (there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    i32, i64, f32 = ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+    lib.qknorm_fwd.argtypes = [_vp, _vp, _vp, _vp, i64, i32, i32, f32, _vp, _vp, _vp]
+    lib.qknorm_fwd.restype = ctypes.c_int
+    lib.qknorm_fwd_ex.argtypes = [_vp, _vp, _vp, _vp, i64, i32, i32, f32, _vp, _vp, _vp, _vp, _vp]
+    lib.qknorm_fwd_ex.restype = ctypes.c_int
+    lib.qknorm_fwd_sharded.argtypes = [_vpp, _vpp, _vpp, _vpp, i32, i64, i32, i32, f32, _vpp, _vpp, _vp]
+    lib.qknorm_fwd_sharded.restype = ctypes.c_int
+    lib.qknorm_fwd_sharded_ex.argtypes = [_vpp, _vpp, _vpp, _vpp, i32, i64, i32, i32, f32, _vpp, _vpp,
+                                          _vp, _vp, _vp, _vp, _vp]
+    lib.qknorm_fwd_sharded_ex.restype = ctypes.c_int
+    lib.qknorm_status_string.argtypes = [ctypes.c_int]
+    lib.qknorm_status_string.restype = ctypes.c_char_p
+    lib.qknorm_last_cuda_error.argtypes = []
+    lib.qknorm_last_cuda_error.restype = ctypes.c_int
+    lib.qknorm_last_variant.argtypes = []
+    lib.qknorm_last_variant.restype = ctypes.c_char_p
+    lib.qknorm_launch_count.argtypes = []
+    lib.qknorm_launch_count.restype = ctypes.c_int64
+    lib.qknorm_version.argtypes = []
+    lib.qknorm_version.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _check(status: int) -> None:
+    if status != QKNORM_OK:
+        lib = load()
+        msg = lib.qknorm_status_string(status).decode()
+        if status == QKNORM_ERR_CUDA:
+            msg += f" (cudaError {lib.qknorm_last_cuda_error()})"
+        raise QKNormError(status, msg)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    return t.data_ptr() or None
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream or None
+
+
+def _expect(t: Optional[torch.Tensor], shape, dtype, what: str) -> None:
+    if t is None:
+        raise QKNormError(QKNORM_ERR_NULL, f"{what} is None")
+    if not t.is_cuda:
+        raise QKNormError(-1, f"{what} must be a CUDA tensor")
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        raise QKNormError(QKNORM_ERR_SHAPE, f"{what}: expected contiguous {dtype} {tuple(shape)}, "
+                                            f"got {t.dtype} {tuple(t.shape)}")
+
+
+def _array(ts: Optional[Sequence[torch.Tensor]], n: int):
+    if ts is None:
+        return None
+    if len(ts) != n:
+        raise QKNormError(QKNORM_ERR_SHARDS, f"expected {n} shards, got {len(ts)}")
+    return (ctypes.c_void_p * n)(*[_ptr(t) for t in ts])
+
+
+def qknorm_fwd(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=None, *,
+               rstd_q=None, rstd_k=None, stream=None):
+    """qknorm_fwd / qknorm_fwd_ex.  q [T,dq], k [T,dk] bf16 CUDA tensors (either may
+    be None to skip that tensor); out_* default to new tensors, and may be the
+    inputs themselves (in place).  Passing rstd_* (fp32 [T]) selects the _ex form.
+    Returns (out_q, out_k)."""
+    lib = load()
+    bf = torch.bfloat16
+    ref = q if q is not None else k
+    if ref is None:
+        raise QKNormError(QKNORM_ERR_NULL, "q and k are both None")
+    T = ref.shape[0]
+    dq = q.shape[1] if q is not None else 0
+    dk = k.shape[1] if k is not None else 0
+    if q is not None:
+        _expect(q, (T, dq), bf, "q")
+        _expect(gamma_q, (dq,), bf, "gamma_q")
+        out_q = torch.empty_like(q) if out_q is None else out_q
+        _expect(out_q, (T, dq), bf, "out_q")
+    if k is not None:
+        _expect(k, (T, dk), bf, "k")
+        _expect(gamma_k, (dk,), bf, "gamma_k")
+        out_k = torch.empty_like(k) if out_k is None else out_k
+        _expect(out_k, (T, dk), bf, "out_k")
+    if rstd_q is not None:
+        _expect(rstd_q, (T,), torch.float32, "rstd_q")
+    if rstd_k is not None:
+        _expect(rstd_k, (T,), torch.float32, "rstd_k")
+    args = [_ptr(q), _ptr(k), _ptr(gamma_q) if q is not None else None,
+            _ptr(gamma_k) if k is not None else None, T, dq, dk, float(eps),
+            _ptr(out_q) if q is not None else None, _ptr(out_k) if k is not None else None]
+    if rstd_q is None and rstd_k is None:
+        _check(lib.qknorm_fwd(*args, _stream(stream)))
+    else:
+        _check(lib.qknorm_fwd_ex(*args, _ptr(rstd_q), _ptr(rstd_k), _stream(stream)))
+    return out_q, out_k
+
+
+def qknorm_fwd_sharded(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: float,
+                       out_q_shards=None, out_k_shards=None, *, partials_q=None, partials_k=None,
+                       rstd_q=None, rstd_k=None, stream=None):
+    """qknorm_fwd_sharded / qknorm_fwd_sharded_ex.  *_shards are lists of S CUDA
+    tensors ([T, dq/S], [T, dk/S], [dq/S], [dk/S]); q_shards or k_shards may be
+    None to skip that tensor.  Passing partials_* (fp32 [S,T]) or rstd_* (fp32
+    [T]) selects the _ex form.  Returns (out_q_shards, out_k_shards)."""
+    lib = load()
+    bf = torch.bfloat16
+    ref = q_shards if q_shards is not None else k_shards
+    if ref is None:
+        raise QKNormError(QKNORM_ERR_NULL, "q_shards and k_shards are both None")
+    S = len(ref)
+    if S < 1:
+        raise QKNormError(QKNORM_ERR_SHARDS, "need at least one shard")
+    T = ref[0].shape[0]
+    wq = q_shards[0].shape[1] if q_shards is not None else 0
+    wk = k_shards[0].shape[1] if k_shards is not None else 0
+
+    def side(xs, gs, outs, w, name):
+        if xs is None:
+            return None, None, None
+        if outs is None:
+            outs = [torch.empty_like(x) for x in xs]
+        if len(xs) != S or len(gs) != S or len(outs) != S:
+            raise QKNormError(QKNORM_ERR_SHARDS, f"{name}: every list must hold {S} shards")
+        for s in range(S):
+            _expect(xs[s], (T, w), bf, f"{name}_shards[{s}]")
+            _expect(gs[s], (w,), bf, f"gamma_{name}_shards[{s}]")
+            _expect(outs[s], (T, w), bf, f"out_{name}_shards[{s}]")
+        return xs, gs, outs
+
+    q_shards, gamma_q_shards, out_q_shards = side(q_shards, gamma_q_shards, out_q_shards, wq, "q")
+    k_shards, gamma_k_shards, out_k_shards = side(k_shards, gamma_k_shards, out_k_shards, wk, "k")
+    for nm, t, shp in (("partials_q", partials_q, (S, T)), ("partials_k", partials_k, (S, T)),
+                       ("rstd_q", rstd_q, (T,)), ("rstd_k", rstd_k, (T,))):
+        if t is not None:
+            _expect(t, shp, torch.float32, nm)
+    args = [_array(q_shards, S), _array(k_shards, S), _array(gamma_q_shards, S), _array(gamma_k_shards, S),
+            S, T, wq * S, wk * S, float(eps), _array(out_q_shards, S), _array(out_k_shards, S)]
+    if all(t is None for t in (partials_q, partials_k, rstd_q, rstd_k)):
+        _check(lib.qknorm_fwd_sharded(*args, _stream(stream)))
+    else:
+        _check(lib.qknorm_fwd_sharded_ex(*args, _ptr(partials_q), _ptr(partials_k), _ptr(rstd_q),
+                                         _ptr(rstd_k), _stream(stream)))
+    return out_q_shards, out_k_shards
+
+
+def last_variant() -> str:
+    return load().qknorm_last_variant().decode()
+
+
+def launch_count() -> int:
+    return int(load().qknorm_launch_count())
+
+
+def version() -> int:
+    return int(load().qknorm_version())

@@ -1,0 +1,57 @@
+// Small device helpers used by every libqknorm kernel: bf16 <-> fp32 on packed
+// words, streaming 128-bit loads/stores.
+#pragma once
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace qknorm {
+
+// A packed word holds two bf16: element 2i in the low half, 2i+1 in the high half.
+__device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// One rounding, to nearest even (cvt.rn.bf16x2.f32); `a` lands in the low half.
+__device__ __forceinline__ uint32_t bf_pack(float a, float b) {
+  __nv_bfloat162 r = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&r);
+}
+
+// Sum of squares of the 8 values of a 16-byte chunk, added to acc (fp32 FMA chain).
+__device__ __forceinline__ float chunk_sumsq(const uint4& v, float acc) {
+  acc = fmaf(bf_lo(v.x), bf_lo(v.x), acc);
+  acc = fmaf(bf_hi(v.x), bf_hi(v.x), acc);
+  acc = fmaf(bf_lo(v.y), bf_lo(v.y), acc);
+  acc = fmaf(bf_hi(v.y), bf_hi(v.y), acc);
+  acc = fmaf(bf_lo(v.z), bf_lo(v.z), acc);
+  acc = fmaf(bf_hi(v.z), bf_hi(v.z), acc);
+  acc = fmaf(bf_lo(v.w), bf_lo(v.w), acc);
+  acc = fmaf(bf_hi(v.w), bf_hi(v.w), acc);
+  return acc;
+}
+
+// (x * gamma) * rstd on one packed word (Algorithm 1: the weight multiply of
+// Phase B, then the scaling of Phase C), rounded once.
+__device__ __forceinline__ uint32_t scale_word(uint32_t x, uint32_t g, float rstd) {
+  return bf_pack((bf_lo(x) * bf_lo(g)) * rstd, (bf_hi(x) * bf_hi(g)) * rstd);
+}
+
+__device__ __forceinline__ uint4 scale_chunk(const uint4& x, const uint4& g, float rstd) {
+  uint4 o;
+  o.x = scale_word(x.x, g.x, rstd);
+  o.y = scale_word(x.y, g.y, rstd);
+  o.z = scale_word(x.z, g.z, rstd);
+  o.w = scale_word(x.w, g.w, rstd);
+  return o;
+}
+
+// Activations are touched once: stream them past the caches.  These are plain
+// coherent accesses (never the read-only path), so an output may alias its input.
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(uint4* p, const uint4& v) { __stcs(p, v); }
+
+// RMS^-1 of Algorithm 1 from the global sum of squares; IEEE divide and sqrt.
+__device__ __forceinline__ float rstd_from_sumsq(float sumsq, int h_total, float eps) {
+  return 1.0f / sqrtf(sumsq / (float)h_total + eps);
+}
+
+}  // namespace qknorm

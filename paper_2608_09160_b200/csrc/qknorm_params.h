@@ -1,0 +1,33 @@
+// Kernel parameter block shared by every kernel variant of libqknorm.
+// Passed by value (__grid_constant__), so the host pointer arrays of the C ABI
+// are consumed during the call and nothing has to be allocated on the device.
+#pragma once
+#include <stdint.h>
+
+namespace qknorm {
+
+constexpr int kMaxShards = 16;   // QKNORM_MAX_SHARDS
+constexpr int kMaxDim = 65536;   // QKNORM_MAX_DIM
+
+// One tensor (Q or K) held as S equal column slices.  S == 1 is the unsharded case.
+struct TensorArgs {
+  const uint16_t* x[kMaxShards];      // X_local of Algorithm 1, slice s: [T, w] bf16
+  const uint16_t* gamma[kMaxShards];  // W_local, slice s: [w] bf16
+  uint16_t* y[kMaxShards];            // Y_local, slice s: [T, w] bf16 (may equal x[s])
+  float* partials;                    // optional [S, T]: Phase A scalar of every slice
+  float* rstd;                        // optional [T]: RMS^-1 of Algorithm 1
+  int d;                              // full width H_total (0 = tensor absent)
+  int w;                              // slice width d / S
+};
+
+struct Params {
+  TensorArgs q, k;
+  long long T;   // tokens
+  int S;         // slices per tensor
+  float eps;
+  // thread grouping of the register-resident kernel: G threads serve one slice
+  int G;         // power of two, >= 16
+  int logG;
+};
+
+}  // namespace qknorm

@@ -24,3 +24,11 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session")
+def libqknorm():
+    """Builds (if stale) and loads the CUDA library; every test that touches the C ABI uses this."""
+    from paper_2608_09160_b200 import binding, build
+    build.build()
+    return binding.load()

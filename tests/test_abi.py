@@ -1,0 +1,107 @@
+"""The C-ABI library loads, exports what include/qknorm.h declares, and rejects
+bad arguments on the host before anything is launched (no GPU needed)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2608_09160_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "qknorm.h")
+
+
+def declared_functions():
+    src = open(HEADER).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(qknorm_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_header_and_binding_agree_on_exports():
+    assert declared_functions() == sorted(binding.EXPORTS)
+
+
+def test_library_exports_every_declared_symbol(libqknorm):
+    for name in declared_functions():
+        assert hasattr(libqknorm, name), name
+    assert libqknorm.qknorm_version() >= 100
+    assert libqknorm.qknorm_status_string(0) == b"QKNORM_OK"
+    for code in range(1, 8):
+        assert libqknorm.qknorm_status_string(code).startswith(b"QKNORM_ERR_")
+    assert libqknorm.qknorm_status_string(99) == b"unknown qknorm status"
+
+
+def test_no_symbol_of_the_oracle_is_linked_in(libqknorm):
+    for name in ("qko_rmsnorm", "qko_rmsnorm_sharded", "qko_f64_to_bf16"):
+        assert not hasattr(libqknorm, name)
+
+
+# Fake device addresses: validation never dereferences them and fails before any launch.
+A, B, C, D, E, F = (0x10000000 + i * 0x1000000 for i in range(6))
+
+
+def fwd(lib, q=A, k=B, gq=C, gk=D, T=4, dq=64, dk=64, eps=1e-6, oq=E, ok=F):
+    return lib.qknorm_fwd(q, k, gq, gk, T, dq, dk, eps, oq, ok, None)
+
+
+def test_unsharded_argument_errors(libqknorm):
+    lib = libqknorm
+    assert fwd(lib, T=0) == binding.QKNORM_OK                   # nothing to do, nothing launched
+    assert fwd(lib, T=-1) == binding.QKNORM_ERR_SHAPE
+    assert fwd(lib, dq=-8) == binding.QKNORM_ERR_SHAPE
+    assert fwd(lib, dq=65536 + 8) == binding.QKNORM_ERR_SHAPE
+    assert fwd(lib, dq=0, dk=0) == binding.QKNORM_ERR_SHAPE
+    assert fwd(lib, eps=-1.0) == binding.QKNORM_ERR_EPS
+    assert fwd(lib, eps=float("nan")) == binding.QKNORM_ERR_EPS
+    assert fwd(lib, q=None) == binding.QKNORM_ERR_NULL
+    assert fwd(lib, gk=None) == binding.QKNORM_ERR_NULL
+    assert fwd(lib, ok=None) == binding.QKNORM_ERR_NULL
+    assert fwd(lib, q=A + 1) == binding.QKNORM_ERR_ALIGN
+    # partial overlap of an output with its input, with the other tensor, with a gamma
+    assert fwd(lib, oq=A + 64) == binding.QKNORM_ERR_ALIAS
+    assert fwd(lib, oq=B) == binding.QKNORM_ERR_ALIAS
+    assert fwd(lib, oq=C) == binding.QKNORM_ERR_ALIAS
+    assert fwd(lib, oq=E, ok=E + 2) == binding.QKNORM_ERR_ALIAS
+
+
+def test_exact_in_place_passes_validation_and_then_needs_a_gpu(libqknorm):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("on a GPU box this call would launch on fake pointers")
+    # out == in is legal; the call gets as far as asking CUDA for the device and fails loudly there
+    assert fwd(libqknorm, oq=A, ok=B) == binding.QKNORM_ERR_CUDA
+    assert libqknorm.qknorm_last_cuda_error() != 0
+    assert fwd(libqknorm, dq=0, q=None, gq=None, oq=None) == binding.QKNORM_ERR_CUDA   # K-only is legal too
+
+
+def sharded(lib, S=4, T=4, dq=64, dk=64, eps=1e-6, q=None, oq=None, k_none=False):
+    arr = ctypes.c_void_p * max(S, 1)
+    n = max(S, 1)
+    mk = lambda base: arr(*[base + i * 0x10000 for i in range(n)])
+    qa = mk(A) if q is None else q
+    oqa = mk(E) if oq is None else oq
+    return lib.qknorm_fwd_sharded(qa, None if k_none else mk(B), mk(C), mk(D), S, T, dq, dk, eps,
+                                  oqa, mk(F), None)
+
+
+def test_sharded_argument_errors(libqknorm):
+    lib = libqknorm
+    assert sharded(lib, S=0) == binding.QKNORM_ERR_SHARDS
+    assert sharded(lib, S=17) == binding.QKNORM_ERR_SHARDS
+    assert sharded(lib, S=3, dq=64) == binding.QKNORM_ERR_SHAPE          # 64 % 3 != 0
+    assert sharded(lib, T=0) == binding.QKNORM_OK
+    assert sharded(lib, k_none=True) == binding.QKNORM_ERR_NULL
+    arr = ctypes.c_void_p * 4
+    assert sharded(lib, q=arr(A, None, A + 0x20000, A + 0x30000)) == binding.QKNORM_ERR_NULL
+    # shard 1's output lands on shard 2's input
+    assert sharded(lib, oq=arr(E, A + 0x20000, E + 0x20000, E + 0x30000)) == binding.QKNORM_ERR_ALIAS
+    # two output shards overlap each other
+    assert sharded(lib, oq=arr(E, E + 16, E + 0x20000, E + 0x30000)) == binding.QKNORM_ERR_ALIAS
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "libqknorm.so"))
+    with pytest.raises(binding.QKNormError, match="no fallback"):
+        binding.load()

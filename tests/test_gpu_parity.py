@@ -1,0 +1,207 @@
+"""GPU parity: libqknorm (through its C ABI) against the fp64 CPU oracle,
+element by element, on the same seeded inputs."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_09160_b200 import binding
+from paper_2608_09160_b200 import workloads as W
+from tests import gpu_harness as H
+
+pytestmark = pytest.mark.gpu
+
+SMALL = W.small_parity_shapes()
+NTHREADS = max(1, min(16, os.cpu_count() or 1))
+
+
+def run_case(w: W.Workload, S: int, *, in_place: bool = False, skew: int = 0, stats: bool = True,
+             force_general: bool = False, monkeypatch=None):
+    """One call through the C ABI with guarded buffers; returns GPU bits and stats."""
+    inp = W.make_inputs(w)
+    T = w.tokens
+    ar = H.arena_for(w, copies=3)
+    dev = {}
+    res = {}
+    if force_general:
+        monkeypatch.setenv("QKNORM_FORCE_VARIANT", "general")
+    kw = dict(skew_elems=skew) if skew else {}
+    has_q, has_k = w.dq > 0, w.dk > 0
+    rq = torch.full((T,), float("nan"), device="cuda") if (stats and has_q) else None
+    rk = torch.full((T,), float("nan"), device="cuda") if (stats and has_k) else None
+    if S == 1:
+        q = H.put(ar, inp["q"], **kw) if has_q else None
+        k = H.put(ar, inp["k"], **kw) if has_k else None
+        gq = H.put(ar, inp["gamma_q"], **kw) if has_q else None
+        gk = H.put(ar, inp["gamma_k"], **kw) if has_k else None
+        oq = q if in_place else (ar.take((T, w.dq), **kw) if has_q else None)
+        ok = k if in_place else (ar.take((T, w.dk), **kw) if has_k else None)
+        binding.qknorm_fwd(q, k, gq, gk, w.eps, oq, ok, rstd_q=rq, rstd_k=rk)
+        torch.cuda.synchronize()
+        res["q"] = H.bits(oq) if has_q else None
+        res["k"] = H.bits(ok) if has_k else None
+        res["pq"] = res["pk"] = None
+    else:
+        def side(x, g, present):
+            if not present:
+                return None, None, None
+            xs = [H.put(ar, p, **kw) for p in W.shard_columns(x, S)]
+            gs = [H.put(ar, p, **kw) for p in W.shard_columns(g, S)]
+            outs = xs if in_place else [ar.take(tuple(p.shape), **kw) for p in xs]
+            return xs, gs, outs
+        qs, gqs, oqs = side(inp["q"], inp["gamma_q"], has_q)
+        ks, gks, oks = side(inp["k"], inp["gamma_k"], has_k)
+        pq = torch.full((S, T), float("nan"), device="cuda") if (stats and has_q) else None
+        pk = torch.full((S, T), float("nan"), device="cuda") if (stats and has_k) else None
+        binding.qknorm_fwd_sharded(qs, ks, gqs, gks, w.eps, oqs, oks, partials_q=pq, partials_k=pk,
+                                   rstd_q=rq, rstd_k=rk)
+        torch.cuda.synchronize()
+        res["q"] = H.bits(W.unshard_columns([o.cpu() for o in oqs])) if has_q else None
+        res["k"] = H.bits(W.unshard_columns([o.cpu() for o in oks])) if has_k else None
+        res["pq"], res["pk"] = pq, pk
+    res["rq"], res["rk"] = rq, rk
+    res["variant"] = binding.last_variant()
+    ar.check()
+    res["inp"] = inp
+    return res
+
+
+def check_against_oracle(w, S, res):
+    inp = res["inp"]
+    ref = H.oracle_unsharded(inp, w.eps, nthreads=NTHREADS)
+    report = {}
+    for name, r, p in (("q", res["rq"], res["pq"]), ("k", res["rk"], res["pk"])):
+        if ref[name] is None:
+            continue
+        report[name] = H.compare_output(res[name], ref[name]["y"], f"{w.name}/S={S}/{name}")
+        if r is not None:
+            H.compare_stat(r, ref[name]["rstd"], f"{w.name}/S={S}/rstd_{name}")
+        if p is not None:
+            xs = [W.bf16_bits(t) for t in W.shard_columns(inp[name], S)]
+            gs = [W.bf16_bits(t) for t in W.shard_columns(inp["gamma_" + name], S)]
+            sh = oracle.rmsnorm_sharded(xs, gs, w.eps, nthreads=NTHREADS)
+            H.compare_stat(p, sh["partials"], f"{w.name}/S={S}/partials_{name}")
+            # the oracle's own sharded form agrees with its unsharded form (same test inputs)
+            assert np.array_equal(np.concatenate(sh["y"], axis=1), ref[name]["y"])
+    return report
+
+
+CASES = [(w, S) for w in SMALL for S in w.shards]
+
+
+@pytest.mark.parametrize("w,S", CASES, ids=[f"{w.name}-S{S}" for w, S in CASES])
+def test_small_shapes_match_oracle(libqknorm, w, S):
+    res = run_case(w, S)
+    check_against_oracle(w, S, res)
+
+
+@pytest.mark.parametrize("w,S", CASES, ids=[f"{w.name}-S{S}" for w, S in CASES])
+def test_small_shapes_in_place(libqknorm, w, S):
+    res = run_case(w, S, in_place=True, stats=False)
+    check_against_oracle(w, S, res)
+
+
+@pytest.mark.parametrize("w,S", CASES[::2], ids=[f"{w.name}-S{S}" for w, S in CASES[::2]])
+def test_general_kernel_matches_oracle(libqknorm, monkeypatch, w, S):
+    res = run_case(w, S, force_general=True, monkeypatch=monkeypatch)
+    assert res["variant"] == "general"
+    check_against_oracle(w, S, res)
+
+
+@pytest.mark.parametrize("skew", [1, 3, 4])
+def test_unaligned_buffers_take_the_general_kernel(libqknorm, skew):
+    w = W.Workload("skewed", tokens=19, dq=1024, dk=256, shards=(1, 4), seed=77)
+    for S in w.shards:
+        res = run_case(w, S, skew=skew)
+        assert res["variant"] == "general"
+        check_against_oracle(w, S, res)
+
+
+def test_vector_kernel_is_the_one_that_runs_on_aligned_shapes(libqknorm):
+    for name in ("s_149", "s_gqa8", "s_t1"):
+        w = next(x for x in SMALL if x.name == name)
+        res = run_case(w, w.shards[0])
+        assert res["variant"] == "rows", (name, res["variant"])
+
+
+def test_results_are_bitwise_reproducible(libqknorm):
+    w = next(x for x in SMALL if x.name == "s_gqa8")
+    a = run_case(w, 8)
+    b = run_case(w, 8)
+    assert np.array_equal(a["q"], b["q"]) and np.array_equal(a["k"], b["k"])
+    assert torch.equal(a["rq"], b["rq"]) and torch.equal(a["pq"], b["pq"])
+
+
+def test_sharded_and_unsharded_agree_within_tolerance(libqknorm):
+    w = W.scaled(W.WORKLOADS["C2"], 64)
+    a = run_case(w, 1)
+    b = run_case(w, 4)
+    for name in ("q", "k"):
+        from tests.util import ordinal_distance
+        assert ordinal_distance(a[name], b[name]).max() <= 2   # each within 1 of the same oracle value
+    check_against_oracle(w, 1, a)
+    check_against_oracle(w, 4, b)
+
+
+def test_closed_form_constant_rows_on_gpu(libqknorm):
+    # y = gamma * c / sqrt(c^2 + eps) for a constant row: exact expectation, no oracle involved
+    T, d = 5, 2048
+    for c, g in ((1.0, 1.0), (-3.0, 0.5), (96.0, 1.25), (2.0 ** -10, -3.0)):
+        q = torch.full((T, d), c, dtype=torch.bfloat16, device="cuda")
+        gam = torch.full((d,), g, dtype=torch.bfloat16, device="cuda")
+        oq, _ = binding.qknorm_fwd(q, None, gam, None, 1e-6)
+        want = oracle.f64_to_bf16(g * c / np.sqrt(c * c + float(np.float32(1e-6))))
+        got = H.bits(oq)
+        from tests.util import ordinal_distance
+        assert ordinal_distance(got, np.full_like(got, want)).max() <= 1
+
+
+def test_zero_rows_nan_rows_and_eps_zero(libqknorm):
+    w = W.Workload("special", tokens=6, dq=1024, dk=128, shards=(1, 4), seed=5)
+    inp = W.make_inputs(w)
+    inp["q"][1].zero_()                       # zero row: finite, signed zeros out
+    inp["q"][2, 17] = float("nan")            # NaN poisons only its row
+    inp["k"][3, 5] = float("inf")
+    for S in w.shards:
+        for eps in (1e-6, 0.0):
+            dq = [t.cuda() for t in W.shard_columns(inp["q"], S)]
+            dk = [t.cuda() for t in W.shard_columns(inp["k"], S)]
+            gq = [t.cuda() for t in W.shard_columns(inp["gamma_q"], S)]
+            gk = [t.cuda() for t in W.shard_columns(inp["gamma_k"], S)]
+            oq, ok = binding.qknorm_fwd_sharded(dq, dk, gq, gk, eps)
+            with np.errstate(all="ignore"):
+                ref = H.oracle_unsharded(inp, eps)
+            H.compare_output(H.bits(W.unshard_columns([o.cpu() for o in oq])), ref["q"]["y"], f"special q S={S} eps={eps}")
+            H.compare_output(H.bits(W.unshard_columns([o.cpu() for o in ok])), ref["k"]["y"], f"special k S={S} eps={eps}")
+
+
+def test_non_default_stream_and_empty_call(libqknorm):
+    w = next(x for x in SMALL if x.name == "s_149")
+    inp = W.make_inputs(w)
+    q, k = inp["q"].cuda(), inp["k"].cuda()
+    gq, gk = inp["gamma_q"].cuda(), inp["gamma_k"].cuda()
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        oq, ok = binding.qknorm_fwd(q, k, gq, gk, w.eps, stream=st)
+    st.synchronize()
+    ref = H.oracle_unsharded(inp, w.eps)
+    H.compare_output(H.bits(oq), ref["q"]["y"], "stream q")
+    H.compare_output(H.bits(ok), ref["k"]["y"], "stream k")
+    n0 = binding.launch_count()
+    e = torch.empty((0, 128), dtype=torch.bfloat16, device="cuda")
+    g = torch.ones((128,), dtype=torch.bfloat16, device="cuda")
+    binding.qknorm_fwd(e, e.clone(), g, g.clone(), 1e-6)
+    assert binding.launch_count() == n0
+
+
+def test_alias_is_rejected_on_real_buffers(libqknorm):
+    buf = torch.zeros((3 * 64 * 128,), dtype=torch.bfloat16, device="cuda")
+    q = buf[: 64 * 128].view(64, 128)
+    out_overlapping = buf[128: 128 + 64 * 128].view(64, 128)
+    g = torch.ones((128,), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.QKNormError) as ei:
+        binding.qknorm_fwd(q, None, g, None, 1e-6, out_overlapping, None)
+    assert ei.value.status == binding.QKNORM_ERR_ALIAS

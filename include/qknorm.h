@@ -118,8 +118,14 @@ const char* qknorm_status_string(int status);
  * library (0 if none). */
 int qknorm_last_cuda_error(void);
 
+/* Debugging aid; SYNCHRONISES the device.  Every wait inside a kernel of this
+ * library is bounded; a wait that ran out makes its CTA leave early and sets a
+ * per-device error word.  This call copies that word to *out (host pointer):
+ * 0 = no wait ever ran out on the current device since the library was loaded. */
+int qknorm_device_error_word(int* out);
+
 /* Name of the kernel variant the last successful call on this thread launched
- * ("rows", "general", "none"); static storage.  For tests and benchmarks. */
+ * ("warp", "ring", "rows", "general", "none"); static storage.  For tests and benchmarks. */
 const char* qknorm_last_variant(void);
 
 /* Number of kernel launches this thread has enqueued through the library. */

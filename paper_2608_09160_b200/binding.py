@@ -22,6 +22,7 @@ EXPORTS = (
     "qknorm_fwd_ex",
     "qknorm_fwd_sharded_ex",
     "qknorm_status_string",
+    "qknorm_device_error_word",
     "qknorm_last_cuda_error",
     "qknorm_last_variant",
     "qknorm_launch_count",
@@ -70,6 +71,8 @@ def load() -> ctypes.CDLL:
     lib.qknorm_fwd_sharded_ex.restype = ctypes.c_int
     lib.qknorm_status_string.argtypes = [ctypes.c_int]
     lib.qknorm_status_string.restype = ctypes.c_char_p
+    lib.qknorm_device_error_word.argtypes = [ctypes.POINTER(ctypes.c_int)]
+    lib.qknorm_device_error_word.restype = ctypes.c_int
     lib.qknorm_last_cuda_error.argtypes = []
     lib.qknorm_last_cuda_error.restype = ctypes.c_int
     lib.qknorm_last_variant.argtypes = []
@@ -207,6 +210,13 @@ def qknorm_fwd_sharded(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: 
         _check(lib.qknorm_fwd_sharded_ex(*args, _ptr(partials_q), _ptr(partials_k), _ptr(rstd_q),
                                          _ptr(rstd_k), _stream(stream)))
     return out_q_shards, out_k_shards
+
+
+def device_error_word() -> int:
+    """Synchronises; 0 unless a bounded in-kernel wait ever ran out on the current device."""
+    out = ctypes.c_int(-1)
+    _check(load().qknorm_device_error_word(ctypes.byref(out)))
+    return int(out.value)
 
 
 def last_variant() -> str:

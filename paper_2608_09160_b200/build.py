@@ -2,7 +2,7 @@
 
     python -m paper_2608_09160_b200.build [--force] [--verbose]
 
-The row kernel is instantiated once per value of NQ in its own translation
+The row kernels are instantiated once per value of N (chunks per thread) in their own translation
 unit, so the objects are compiled in parallel and linked into one shared
 library next to this file.
 """
@@ -23,7 +23,8 @@ INCLUDE = os.path.join(os.path.dirname(PKG_DIR), "include")
 BUILD_DIR = os.path.join(PKG_DIR, "build")
 LIB_PATH = os.path.join(PKG_DIR, "libqknorm.so")
 
-ROWS_NQ = (0, 1, 2, 3, 4, 5, 6, 8)
+CHUNKS_PER_THREAD = (1, 2, 3, 4, 6, 8)          # row / ring kernels
+CHUNK_SLOTS_PER_LANE = tuple(range(4, 44, 4))    # warp-per-row kernel
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
@@ -43,8 +44,10 @@ def _nvcc() -> str:
 def _units() -> List[Tuple[str, str, List[str]]]:
     """(object name, source, extra flags)"""
     units = [("qknorm_api.o", os.path.join(CSRC, "qknorm_api.cu"), [])]
-    for n in ROWS_NQ:
-        units.append((f"qknorm_rows_nq{n}.o", os.path.join(CSRC, "qknorm_rows_inst.cu"), [f"-DQKNORM_NQ={n}"]))
+    for n in CHUNKS_PER_THREAD:
+        units.append((f"qknorm_rows_n{n}.o", os.path.join(CSRC, "qknorm_rows_inst.cu"), [f"-DQKNORM_N={n}"]))
+    for l in CHUNK_SLOTS_PER_LANE:
+        units.append((f"qknorm_warp_l{l}.o", os.path.join(CSRC, "qknorm_warp_inst.cu"), [f"-DQKNORM_L={l}"]))
     return units
 
 

@@ -10,40 +10,70 @@
 #include "../../include/qknorm.h"
 #include "qknorm_general.cuh"
 #include "qknorm_params.h"
+#include "qknorm_ring.cuh"
 #include "qknorm_rows.cuh"
+#include "qknorm_warp.cuh"
 
 namespace qknorm {
 
-// per-NQ factories, defined in qknorm_rows_inst.cu
-#define QKNORM_DECL_TP(n) RowsKernel rows_throughput_nq##n(int nk);
-#define QKNORM_DECL_LAT(n) RowsKernel rows_latency_nq##n(int nk);
-QKNORM_DECL_TP(0) QKNORM_DECL_TP(1) QKNORM_DECL_TP(2) QKNORM_DECL_TP(3)
-QKNORM_DECL_TP(4) QKNORM_DECL_TP(5) QKNORM_DECL_TP(6) QKNORM_DECL_TP(8)
-QKNORM_DECL_LAT(0) QKNORM_DECL_LAT(1) QKNORM_DECL_LAT(2) QKNORM_DECL_LAT(4)
+// per-N factories, defined in qknorm_rows_inst.cu (one translation unit per N)
+#define QKNORM_DECL_N(n)        \
+  RowsKernel rows_kernel_n##n(); \
+  RingKernel ring_kernel_n##n();
+QKNORM_DECL_N(1) QKNORM_DECL_N(2) QKNORM_DECL_N(3) QKNORM_DECL_N(4) QKNORM_DECL_N(6) QKNORM_DECL_N(8)
 
-RowsKernel rows_kernel_throughput(int nq, int nk) {
-  switch (nq) {
-    case 0: return rows_throughput_nq0(nk);
-    case 1: return rows_throughput_nq1(nk);
-    case 2: return rows_throughput_nq2(nk);
-    case 3: return rows_throughput_nq3(nk);
-    case 4: return rows_throughput_nq4(nk);
-    case 5: return rows_throughput_nq5(nk);
-    case 6: return rows_throughput_nq6(nk);
-    case 8: return rows_throughput_nq8(nk);
+RowsKernel rows_kernel_for(int n) {
+  switch (n) {
+    case 1: return rows_kernel_n1();
+    case 2: return rows_kernel_n2();
+    case 3: return rows_kernel_n3();
+    case 4: return rows_kernel_n4();
+    case 6: return rows_kernel_n6();
+    case 8: return rows_kernel_n8();
     default: return nullptr;
   }
 }
 
-RowsKernel rows_kernel_latency(int nq, int nk) {
-  switch (nq) {
-    case 0: return rows_latency_nq0(nk);
-    case 1: return rows_latency_nq1(nk);
-    case 2: return rows_latency_nq2(nk);
-    case 4: return rows_latency_nq4(nk);
+RingKernel ring_kernel_for(int n) {
+  switch (n) {
+    case 1: return ring_kernel_n1();
+    case 2: return ring_kernel_n2();
+    case 3: return ring_kernel_n3();
+    case 4: return ring_kernel_n4();
+    case 6: return ring_kernel_n6();
+    case 8: return ring_kernel_n8();
     default: return nullptr;
   }
 }
+
+// per-L factories, defined in qknorm_warp_inst.cu (one translation unit per L)
+#define QKNORM_DECL_L(l) WarpKernel warp_kernel_l##l(bool exact);
+QKNORM_DECL_L(4) QKNORM_DECL_L(8) QKNORM_DECL_L(12) QKNORM_DECL_L(16) QKNORM_DECL_L(20)
+QKNORM_DECL_L(24) QKNORM_DECL_L(28) QKNORM_DECL_L(32) QKNORM_DECL_L(36) QKNORM_DECL_L(40)
+
+int warp_round_up_l(int n) {
+  if (n < 1 || n > 40) return -1;
+  return ((n + 3) / 4) * 4;
+}
+
+WarpKernel warp_kernel_for(int l, bool exact) {
+  switch (l) {
+    case 4: return warp_kernel_l4(exact);
+    case 8: return warp_kernel_l8(exact);
+    case 12: return warp_kernel_l12(exact);
+    case 16: return warp_kernel_l16(exact);
+    case 20: return warp_kernel_l20(exact);
+    case 24: return warp_kernel_l24(exact);
+    case 28: return warp_kernel_l28(exact);
+    case 32: return warp_kernel_l32(exact);
+    case 36: return warp_kernel_l36(exact);
+    case 40: return warp_kernel_l40(exact);
+    default: return nullptr;
+  }
+}
+
+// Set by a ring kernel whose bounded wait ran out (0 = never happened).
+__device__ int g_ring_error = 0;
 
 namespace {
 
@@ -54,6 +84,9 @@ thread_local long long tl_launches = 0;
 struct DeviceInfo {
   bool known = false;
   int sm_count = 0;
+  int smem_per_sm = 0;       // bytes
+  int smem_per_block = 0;    // opt-in maximum, bytes
+  int* ring_error = nullptr; // device address of g_ring_error on this device
 };
 constexpr int kMaxDevices = 64;
 DeviceInfo g_devices[kMaxDevices];
@@ -64,8 +97,8 @@ int set_cuda_error(cudaError_t e) {
   return QKNORM_ERR_CUDA;
 }
 
-// SM count of the current device, cached.
-int current_sm_count(int* out) {
+// Facts about the current device, cached.
+int current_device(const DeviceInfo** out) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return set_cuda_error(e);
@@ -77,9 +110,16 @@ int current_sm_count(int* out) {
     e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return set_cuda_error(e);
     d.sm_count = n;
+    e = cudaDeviceGetAttribute(&d.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
+    if (e != cudaSuccess) return set_cuda_error(e);
+    e = cudaDeviceGetAttribute(&d.smem_per_block, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) return set_cuda_error(e);
+    // the symbol's name is only a host-side handle: ask for its address on this device
+    e = cudaGetSymbolAddress((void**)&d.ring_error, g_ring_error);
+    if (e != cudaSuccess) return set_cuda_error(e);
     d.known = true;
   }
-  *out = d.sm_count;
+  *out = &d;
   return QKNORM_OK;
 }
 
@@ -145,45 +185,70 @@ int env_int(const char* name, int fallback) {
 }
 
 struct RowsPlan {
-  RowsKernel fn = nullptr;
-  int threads = 0, G = 0, logG = 0, nq = 0, nk = 0;
+  int n = 0;        // 16-byte chunks per thread
+  int threads = 0;  // CTA size
+  int log_sub = 5;  // lane-group size (log2)
+  int Gq = 0, Gk = 0;
 };
 
-// Pick the thread grouping (G threads per slice) of the register-resident kernel.
-//  throughput: CTAs of <= 256 threads, as few wasted lanes as possible;
-//  latency (few tokens): CTAs of <= 512 threads and as few chunks per thread as possible,
-//  so that one load round trip covers the row.
+inline int round_up(int v, int m) { return ((v + m - 1) / m) * m; }
+
+// Thread layout of the vectorised kernels (qknorm_rowmap.cuh): N chunks per
+// thread, G_q / G_k threads per Q / K slice, lane groups of 16 or 32.
+//  throughput: wide CTAs with few chunks per thread (many warps hide the latency
+//              of the per-token reduction), as few idle lanes as possible;
+//  latency (few tokens): as few chunks per thread as possible, so that one load
+//              round trip covers the row.
 bool plan_rows(const Params& P, bool latency, RowsPlan* plan) {
   const int cq = P.q.d ? P.q.w / 8 : 0, ck = P.k.d ? P.k.w / 8 : 0;
-  const int max_threads = latency ? 512 : 256;
-  const int forced = env_int("QKNORM_FORCE_G", 0);
+  const int force_n = env_int("QKNORM_FORCE_N", 0);
+  const int force_sub = env_int("QKNORM_FORCE_SUB", 0);
+  const int ns[] = {1, 2, 3, 4, 6, 8};
   double best_cost = 1e30;
   bool found = false;
-  for (int logG = 4; logG <= 9; ++logG) {
-    const int G = 1 << logG;
-    if (forced && G != forced) continue;
-    const int threads = ((P.S * G + 31) / 32) * 32;
-    if (threads > max_threads) continue;
-    const int nq = rows_round_up_n((cq + G - 1) / G, latency), nk = rows_round_up_n((ck + G - 1) / G, latency);
-    if (nq < 0 || nk < 0) continue;
-    RowsKernel fn = latency ? rows_kernel_latency(nq, nk) : rows_kernel_throughput(nq, nk);
-    if (!fn) continue;
-    // lanes issued per useful chunk; latency mode adds a strong preference for few chunks per thread
-    double cost = (double)(nq + nk) * threads / (double)((cq + ck) * P.S);
-    if (latency) cost += 4.0 * (nq + nk);
-    else cost -= 1e-3 * logG;  // tie: wider groups, fewer registers
-    if (cost < best_cost) {
-      best_cost = cost;
-      *plan = RowsPlan{fn, threads, G, logG, nq, nk};
-      found = true;
+  for (int n : ns) {
+    if (force_n && n != force_n) continue;
+    for (int log_sub = 5; log_sub >= 4; --log_sub) {
+      const int sub = 1 << log_sub;
+      if (force_sub && sub != force_sub) continue;
+      const int Gq = cq ? round_up((cq + n - 1) / n, sub) : 0;
+      const int Gk = ck ? round_up((ck + n - 1) / n, sub) : 0;
+      const int threads = round_up(P.S * (Gq + Gk), 32);
+      if (threads > max_threads_for(n)) continue;
+      if (P.S * (Gq + Gk) / sub > kMaxSlots) continue;
+      // Estimated warp instructions per token: per chunk position ~45, per token and
+      // thread ~60 plus the slots it has to add up.  Decode sizes instead want the
+      // shortest dependent chain (few chunks per thread), whatever the lane count.
+      const int warps = threads / 32;
+      const int slots = P.S * (Gq > Gk ? Gq : Gk) / sub;
+      double cost = latency ? (double)n * 1000.0 + warps : (double)warps * (45.0 * n + 60.0 + 2.0 * slots);
+      if (log_sub == 4) cost *= 1.001;  // tie: full-warp groups (fewer slots to add up)
+      if (cost < best_cost) {
+        best_cost = cost;
+        plan->n = n;
+        plan->threads = threads;
+        plan->log_sub = log_sub;
+        plan->Gq = Gq;
+        plan->Gk = Gk;
+        found = true;
+      }
     }
   }
   return found;
 }
 
+void apply_plan(Params& P, const RowsPlan& plan) {
+  P.log_sub = plan.log_sub;
+  P.q.G = plan.Gq;
+  P.q.first_thread = 0;
+  P.k.G = plan.Gk;
+  P.k.first_thread = P.S * plan.Gq;
+}
+
 struct OccKey {
   const void* fn;
   int threads;
+  int smem;
   int dev;
   int blocks;
 };
@@ -193,66 +258,203 @@ int g_occ_n = 0;
 std::mutex g_occ_mutex;
 
 // Resident CTAs per SM for (kernel, CTA size) on the current device: B_res of Section III-D.
-int resident_blocks(const void* fn, int threads, int* out) {
+int resident_blocks(const void* fn, int threads, int smem, int* out) {
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return set_cuda_error(e);
   std::lock_guard<std::mutex> lock(g_occ_mutex);
   for (int i = 0; i < g_occ_n; ++i)
-    if (g_occ[i].fn == fn && g_occ[i].threads == threads && g_occ[i].dev == dev) {
+    if (g_occ[i].fn == fn && g_occ[i].threads == threads && g_occ[i].smem == smem && g_occ[i].dev == dev) {
       *out = g_occ[i].blocks;
       return QKNORM_OK;
     }
   int blocks = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, fn, threads, 0);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&blocks, fn, threads, smem);
   if (e != cudaSuccess) return set_cuda_error(e);
   if (blocks < 1) blocks = 1;
-  if (g_occ_n < kOccCache) g_occ[g_occ_n++] = OccKey{fn, threads, dev, blocks};
+  if (g_occ_n < kOccCache) g_occ[g_occ_n++] = OccKey{fn, threads, smem, dev, blocks};
   *out = blocks;
   return QKNORM_OK;
 }
 
-int launch(Params& P, cudaStream_t stream) {
-  int sms = 0;
-  int rc = current_sm_count(&sms);
+// Largest dynamic shared memory a kernel has been allowed so far, per (kernel, device).
+struct SmemKey {
+  const void* fn;
+  int dev;
+  int bytes;
+};
+SmemKey g_smem[kOccCache];
+int g_smem_n = 0;
+
+int allow_dynamic_smem(const void* fn, int bytes) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return set_cuda_error(e);
+  std::lock_guard<std::mutex> lock(g_occ_mutex);
+  for (int i = 0; i < g_smem_n; ++i)
+    if (g_smem[i].fn == fn && g_smem[i].dev == dev) {
+      if (g_smem[i].bytes >= bytes) return QKNORM_OK;
+      e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+      if (e != cudaSuccess) return set_cuda_error(e);
+      g_smem[i].bytes = bytes;
+      return QKNORM_OK;
+    }
+  e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return set_cuda_error(e);
+  if (g_smem_n < kOccCache) g_smem[g_smem_n++] = SmemKey{fn, dev, bytes};
+  return QKNORM_OK;
+}
+
+int finish_launch(const char* variant) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return set_cuda_error(e);
+  tl_variant = variant;
+  ++tl_launches;
+  return QKNORM_OK;
+}
+
+// The TMA ring kernel (prefill sizes).  Returns QKNORM_OK with *done = false when
+// the shape does not fit it and another variant should run.
+int launch_ring(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* done) {
+  *done = false;
+  RowsPlan plan;
+  if (!plan_rows(P, /*latency=*/false, &plan)) return QKNORM_OK;
+  RingKernel fn = ring_kernel_for(plan.n);
+  if (!fn) return QKNORM_OK;
+  const int row_bytes = (P.q.d + P.k.d) * 2;
+  const int stage_bytes = ((row_bytes + 16 + 127) / 128) * 128;  // the row, then >= 16 bytes of zeros
+  // Split the SM's shared memory between `ctas` resident CTAs, each with as deep a ring as fits.
+  int ctas = env_int("QKNORM_CTAS_PER_SM", 0);
+  if (ctas < 1) {
+    ctas = 2048 / plan.threads;  // as many as the SM's thread slots allow ...
+    if (ctas > 3) ctas = 3;
+    if (ctas < 1) ctas = 1;
+  }
+  const int reserve = 2048;  // static shared memory + the per-CTA system reservation
+  int nst = 0;
+  for (; ctas >= 1; --ctas) {   // ... as long as every CTA still gets a ring of >= 3 stages
+    int budget = dev.smem_per_sm / ctas - reserve;
+    if (budget > dev.smem_per_block - reserve) budget = dev.smem_per_block - reserve;
+    nst = budget / stage_bytes;
+    if (nst >= 3 || ctas == 1) break;
+  }
+  const int forced = env_int("QKNORM_RING_STAGES", 0);
+  if (forced > 0 && forced < nst) nst = forced;
+  if (nst > kRingMaxStages) nst = kRingMaxStages;
+  if (nst < 2) return QKNORM_OK;
+  const int smem = nst * stage_bytes;
+  int rc = allow_dynamic_smem((const void*)fn, smem);
   if (rc != QKNORM_OK) return rc;
+  int bres = 1;
+  rc = resident_blocks((const void*)fn, plan.threads, smem, &bres);
+  if (rc != QKNORM_OK) return rc;
+  if (bres > ctas) bres = ctas;
+  long long grid = (long long)bres * dev.sm_count;  // bounded grid of co-resident CTAs
+  if (grid > P.T) grid = P.T;
+  apply_plan(P, plan);
+  fn<<<(unsigned)grid, plan.threads, smem, stream>>>(P, nst, stage_bytes, dev.ring_error);
+  rc = finish_launch("ring");
+  *done = rc == QKNORM_OK;
+  return rc;
+}
+
+// The warp-per-token kernel (prefill sizes, gathered rows of up to 40 chunks per lane).
+int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* done) {
+  *done = false;
+  int log_g = 5;
+  while ((P.S << log_g) > 32) --log_g;  // g = largest power of two <= 32 / S
+  const int g = 1 << log_g;
+  const int cq = P.q.d ? P.q.w / 8 : 0, ck = P.k.d ? P.k.w / 8 : 0;
+  WarpArgs wa;
+  wa.log_g = log_g;
+  wa.nq = (cq + g - 1) / g;
+  wa.nk = (ck + g - 1) / g;
+  wa.nq4 = round_up(wa.nq, 4);
+  const int l = warp_round_up_l(wa.nq4 + wa.nk);
+  if (l < 0) return QKNORM_OK;
+  const bool exact = (P.S << log_g) == 32 && cq % g == 0 && ck % g == 0 && wa.nq % 4 == 0 && wa.nk % 4 == 0;
+  WarpKernel fn = warp_kernel_for(l, exact);
+  if (!fn) return QKNORM_OK;
+  // stage layout: Q slices, K slices (each slice row followed by the bank skew), 16 zero bytes
+  const int skew = (P.S > 1 && g < 8) ? g * 16 : 0;
+  wa.q_slice_stride = cq ? P.q.w * 2 + skew : 0;
+  wa.k_slice_stride = ck ? P.k.w * 2 + skew : 0;
+  wa.k_base = P.S * wa.q_slice_stride;
+  wa.zero_off = wa.k_base + P.S * wa.k_slice_stride;
+  wa.stage_bytes = round_up(wa.zero_off + 16, 128);
+  wa.error_word = dev.ring_error;
+  // One row per warp is always in flight.  Measured on B200: throughput peaks when
+  // about 76 KB of rows are in flight per SM and falls off slowly beyond that.
+  int per_sm = (76 * 1024 + wa.stage_bytes / 2) / wa.stage_bytes;
+  if (per_sm < 2) per_sm = 2;
+  if (per_sm > 16) per_sm = 16;
+  int ctas_per_sm = per_sm > kWarpMaxCtaWarps ? 2 : 1;
+  int warps = env_int("QKNORM_WARPS", (per_sm + ctas_per_sm - 1) / ctas_per_sm);
+  if (warps < 1) warps = 1;
+  if (warps > kWarpMaxCtaWarps) warps = kWarpMaxCtaWarps;
+  while (warps > 1 && warps * wa.stage_bytes + l * 512 + 1024 > dev.smem_per_block) --warps;
+  const int smem = warps * wa.stage_bytes;
+  if (smem + l * 512 + 1024 > dev.smem_per_block) return QKNORM_OK;
+  int rc = allow_dynamic_smem((const void*)fn, smem);
+  if (rc != QKNORM_OK) return rc;
+  int bres = 1;
+  rc = resident_blocks((const void*)fn, warps * 32, smem, &bres);
+  if (rc != QKNORM_OK) return rc;
+  const int cap = env_int("QKNORM_CTAS_PER_SM", ctas_per_sm);
+  if (cap > 0 && cap < bres) bres = cap;
+  long long grid = (long long)bres * dev.sm_count;  // bounded grid of co-resident CTAs
+  const long long needed = (P.T + warps - 1) / warps;
+  if (grid > needed) grid = needed;
+  fn<<<(unsigned)grid, warps * 32, smem, stream>>>(P, wa);
+  rc = finish_launch("warp");
+  *done = rc == QKNORM_OK;
+  return rc;
+}
+
+int launch(Params& P, cudaStream_t stream) {
+  const DeviceInfo* dev = nullptr;
+  int rc = current_device(&dev);
+  if (rc != QKNORM_OK) return rc;
+  const int sms = dev->sm_count;
   const char* force = getenv("QKNORM_FORCE_VARIANT");
   const bool force_general = force && strcmp(force, "general") == 0;
+  const bool force_rows = force && strcmp(force, "rows") == 0;
+  const bool force_ring = force && strcmp(force, "ring") == 0;
 
   if (!force_general && vector_path_ok(P)) {
     const bool latency = P.T < 4LL * sms;
+    if (!latency && !force_rows && !force_ring) {
+      bool done = false;
+      rc = launch_warp(P, *dev, stream, &done);
+      if (rc != QKNORM_OK || done) return rc;
+    }
+    if (!latency && !force_rows) {
+      bool done = false;
+      rc = launch_ring(P, *dev, stream, &done);
+      if (rc != QKNORM_OK || done) return rc;
+    }
     RowsPlan plan;
     if (plan_rows(P, latency, &plan)) {
-      P.G = plan.G;
-      P.logG = plan.logG;
+      RowsKernel fn = rows_kernel_for(plan.n);
       int bres = 1;
-      rc = resident_blocks((const void*)plan.fn, plan.threads, &bres);
+      rc = resident_blocks((const void*)fn, plan.threads, 0, &bres);
       if (rc != QKNORM_OK) return rc;
       const int cap = env_int("QKNORM_CTAS_PER_SM", 0);
       if (cap > 0 && cap < bres) bres = cap;
       long long grid = (long long)bres * sms;  // bounded grid of co-resident CTAs
       if (grid > P.T) grid = P.T;
-      plan.fn<<<(unsigned)grid, plan.threads, 0, stream>>>(P);
-      cudaError_t e = cudaGetLastError();
-      if (e != cudaSuccess) return set_cuda_error(e);
-      tl_variant = "rows";
-      ++tl_launches;
-      return QKNORM_OK;
+      apply_plan(P, plan);
+      fn<<<(unsigned)grid, plan.threads, 0, stream>>>(P);
+      return finish_launch("rows");
     }
   }
-  {
-    int bres = 1;
-    rc = resident_blocks((const void*)general_kernel, kGeneralThreads, &bres);
-    if (rc != QKNORM_OK) return rc;
-    long long grid = (long long)bres * sms;
-    if (grid > 2 * P.T) grid = 2 * P.T;
-    general_kernel<<<(unsigned)grid, kGeneralThreads, 0, stream>>>(P);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return set_cuda_error(e);
-    tl_variant = "general";
-    ++tl_launches;
-  }
-  return QKNORM_OK;
+  int bres = 1;
+  rc = resident_blocks((const void*)general_kernel, kGeneralThreads, 0, &bres);
+  if (rc != QKNORM_OK) return rc;
+  long long grid = (long long)bres * sms;
+  if (grid > 2 * P.T) grid = 2 * P.T;
+  general_kernel<<<(unsigned)grid, kGeneralThreads, 0, stream>>>(P);
+  return finish_launch("general");
 }
 
 // Shared body of the four entry points.  Pointer arrays are host arrays of S entries.
@@ -273,8 +475,7 @@ int run(const void* const* q, const void* const* k, const void* const* gq, const
   P.T = T;
   P.S = S;
   P.eps = eps;
-  P.G = 32;
-  P.logG = 5;
+  P.log_sub = 5;
   struct Side {
     TensorArgs* a;
     const void* const* x;
@@ -287,6 +488,7 @@ int run(const void* const* q, const void* const* k, const void* const* gq, const
   for (Side& sd : sides) {
     sd.a->d = sd.d;
     sd.a->w = sd.d / S;
+    sd.a->inv_d = sd.d ? 1.0f / (float)sd.d : 0.0f;
     if (sd.d == 0) continue;
     for (int s = 0; s < S; ++s) {
       if (!sd.x[s] || !sd.g[s] || !sd.y[s]) return QKNORM_ERR_NULL;
@@ -351,6 +553,13 @@ const char* qknorm_status_string(int status) {
     case QKNORM_ERR_CUDA: return "QKNORM_ERR_CUDA: a CUDA call failed";
     default: return "unknown qknorm status";
   }
+}
+
+int qknorm_device_error_word(int* out) {
+  if (!out) return QKNORM_ERR_NULL;
+  cudaError_t e = cudaMemcpyFromSymbol(out, qknorm::g_ring_error, sizeof(int));
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  return QKNORM_OK;
 }
 
 int qknorm_last_cuda_error(void) { return qknorm::tl_cuda_error; }

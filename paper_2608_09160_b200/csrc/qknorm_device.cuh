@@ -44,6 +44,31 @@ __device__ __forceinline__ uint4 scale_chunk(const uint4& x, const uint4& g, flo
   return o;
 }
 
+// Mixed-precision FMA of sm_100 (PTX fma.rn.f32.bf16): d = a*b + c with a, b the
+// bf16 halves of packed words and c, d fp32.  The product of two bf16 values is
+// exact in fp32, so this rounds exactly like widening first and using an fp32
+// FMA, without the two widening instructions per word.
+__device__ __forceinline__ void fma_bf16x2_sq(uint32_t x, float& acc_lo, float& acc_hi) {
+  asm("{\n\t.reg .b16 lo, hi;\n\t"
+      "mov.b32 {lo, hi}, %2;\n\t"
+      "fma.rn.f32.bf16 %0, lo, lo, %0;\n\t"
+      "fma.rn.f32.bf16 %1, hi, hi, %1;\n\t}"
+      : "+f"(acc_lo), "+f"(acc_hi)
+      : "r"(x));
+}
+// (x_lo * g_lo, x_hi * g_hi) in fp32, exact; the addend is -0 so that a product of -0 keeps its sign.
+__device__ __forceinline__ float2 mul_bf16x2(uint32_t x, uint32_t g) {
+  float2 p;
+  asm("{\n\t.reg .b16 xl, xh, gl, gh;\n\t"
+      "mov.b32 {xl, xh}, %2;\n\t"
+      "mov.b32 {gl, gh}, %3;\n\t"
+      "fma.rn.f32.bf16 %0, xl, gl, 0f80000000;\n\t"
+      "fma.rn.f32.bf16 %1, xh, gh, 0f80000000;\n\t}"
+      : "=f"(p.x), "=f"(p.y)
+      : "r"(x), "r"(g));
+  return p;
+}
+
 // Activations are touched once: stream them past the caches.  These are plain
 // coherent accesses (never the read-only path), so an output may alias its input.
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }

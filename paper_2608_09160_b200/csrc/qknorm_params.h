@@ -8,6 +8,7 @@ namespace qknorm {
 
 constexpr int kMaxShards = 16;   // QKNORM_MAX_SHARDS
 constexpr int kMaxDim = 65536;   // QKNORM_MAX_DIM
+constexpr int kMaxSlots = 64;    // shared-memory partial sums per CTA (one per 16- or 32-lane group)
 
 // One tensor (Q or K) held as S equal column slices.  S == 1 is the unsharded case.
 struct TensorArgs {
@@ -18,6 +19,10 @@ struct TensorArgs {
   float* rstd;                        // optional [T]: RMS^-1 of Algorithm 1
   int d;                              // full width H_total (0 = tensor absent)
   int w;                              // slice width d / S
+  float inv_d;                        // 1 / H_total
+  // thread layout of the vectorised kernels (see qknorm_rowmap.cuh)
+  int G;                              // threads serving one slice of this tensor (multiple of `sub`)
+  int first_thread;                   // first thread of this tensor's block of S*G threads
 };
 
 struct Params {
@@ -25,9 +30,7 @@ struct Params {
   long long T;   // tokens
   int S;         // slices per tensor
   float eps;
-  // thread grouping of the register-resident kernel: G threads serve one slice
-  int G;         // power of two, >= 16
-  int logG;
+  int log_sub;   // 4 or 5: lanes that reduce together by shuffle (16 or 32)
 };
 
 }  // namespace qknorm

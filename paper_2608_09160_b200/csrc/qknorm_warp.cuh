@@ -1,0 +1,251 @@
+// Prefill kernel: one warp per token, fed by the TMA unit.
+//
+// Every warp owns ONE shared-memory stage and one mbarrier.  The stage holds the
+// warp's current token as the gathered row (Q slices, then K slices).  Per token:
+//
+//   wait for the stage  ->  drain it into registers (every lane pulls its 16-byte
+//   chunks, up to L of them)  ->  per-slice sums of squares with shuffles only
+//   ->  as soon as that reduction is done every lane has consumed the stage, so
+//   the warp re-arms it with its NEXT token (2*S bulk copies, one per slice row)
+//   ->  slices' scalars added in ascending slice order, RMS^-1, (x*gamma)*RMS^-1,
+//   streaming 16-byte stores straight from registers.
+//
+// So each warp always has its next row in flight while it works on the current
+// one (about 18-20 KB per warp, 8 warps per SM), there is no block-level barrier
+// in the token loop, and the instructions per token that are not per-chunk work
+// (shuffles, rsqrt, barrier wait, TMA issue) are spread over the whole row instead
+// of a few chunks per thread.  That matters: this op has to push ~1.6e12
+// elements/s through 148 SMs, so the instruction issue rate bounds it as much as
+// DRAM does.
+//
+// Lane layout.  The 32 lanes are cut into S groups of g lanes (g = largest power
+// of two <= 32/S); group s serves slice s ("rank" s of Algorithm 1) of both
+// tensors.  Lane l of a group owns chunks l, l+g, l+2g, ... of its Q slice row
+// (chunk slots 0 .. nq-1) and of its K slice row (slots nq4 .. nq4+nk-1, nq4 = nq
+// rounded up to a multiple of 4).  Because the row arrives through shared memory,
+// global traffic is whole slice rows whatever S is.  The slice scalar S_local is
+// the lane's own sum plus a log2(g)-step shuffle tree (Phase A); the scalars are
+// added in ascending slice order with S broadcasts (the P2P-reduction line of
+// Phase B); RMS^-1 = rsqrt(S_global / H_total + eps); y = (x*gamma)*RMS^-1,
+// rounded once (Phases B/C).
+//
+// Shared memory.  Slice s of a tensor starts at s * (slice bytes + skew) inside
+// the stage; the skew (g*16 bytes when g < 8) puts the lane groups that read in
+// the same quarter-warp on different banks.  16 bytes of zeros close the stage: a
+// chunk slot a lane does not have is read from there, so loads need no bounds
+// test and add nothing to the sums.  gamma is staged once per CTA as
+// [chunk slot][lane], conflict-free for every warp.
+//
+// In-place calls are safe: a row is completely in registers before any of it is
+// overwritten, and the only other row the warp touches is its next one.
+// Every mbarrier wait is bounded (about one second); a wait that runs out records
+// an error word and the warp leaves.
+#pragma once
+#include "qknorm_ring.cuh"
+#include "qknorm_rowmap.cuh"
+
+namespace qknorm {
+
+constexpr int kWarpMaxCtaWarps = 8;  // the CTA size is a launch parameter: 1..8 warps
+// registers are shaped for this many resident CTAs of 8 warps
+__host__ __device__ constexpr int warp_min_blocks(int l) { return l <= 8 ? 4 : (l <= 16 ? 2 : 1); }
+
+struct WarpArgs {
+  int log_g;            // log2 of the lanes per slice
+  int nq, nk;           // chunk slots in use per lane for the Q part / the K part
+  int nq4;              // first K slot (nq rounded up to a multiple of 4)
+  int stage_bytes;      // bytes of one warp's stage (multiple of 128)
+  int q_slice_stride;   // bytes between consecutive Q slices inside a stage (slice bytes + skew)
+  int k_slice_stride;
+  int k_base;           // byte offset of the K part inside a stage
+  int zero_off;         // byte offset of the 16 zero bytes
+  int* error_word;
+};
+
+// EXACT: every lane has all nq / nk chunk slots (S*g == 32 and the slice rows are
+// whole multiples of g chunks), so the stores need no per-lane test either.
+template <int L, bool EXACT>
+__global__ void __launch_bounds__(kWarpMaxCtaWarps * 32, warp_min_blocks(L))
+warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs wa) {
+  extern __shared__ __align__(128) unsigned char warp_smem[];  // one stage per warp
+  __shared__ uint4 gsm[L][32];
+  __shared__ __align__(8) unsigned long long bars[kWarpMaxCtaWarps];
+
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int g = 1 << wa.log_g;
+  const int s = lane >> wa.log_g;
+  const int l = lane & (g - 1);
+  const bool active = s < P.S;
+  const int ss = active ? s : 0;
+  const int cq = P.q.w >> 3, ck = P.k.w >> 3;  // 16-byte chunks per slice row
+  const int nvq = EXACT ? wa.nq : ((active && l < cq) ? (cq - l + g - 1) / g : 0);
+  const int nvk = EXACT ? wa.nk : ((active && l < ck) ? (ck - l + g - 1) / g : 0);
+  const int n_slots = wa.nq4 + wa.nk;  // uniform
+
+  unsigned char* stage = warp_smem + (size_t)warp * wa.stage_bytes;
+  const uint32_t stage_u32 = ptx::smem_u32(stage);
+  const uint32_t bar = ptx::smem_u32(&bars[warp]);
+  if (lane == 0) {
+    ptx::mbar_init(bar, 1u);
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+    *reinterpret_cast<uint4*>(stage + wa.zero_off) = make_uint4(0u, 0u, 0u, 0u);
+  }
+  // ---- who issues which bulk copy: lane i < S the Q slice row i, lane S+i the K slice row i ----
+  const bool issue_q = lane < P.S;
+  const int is = issue_q ? lane : lane - P.S;
+  uint32_t my_bytes = 0, my_dst = 0;
+  const unsigned char* my_src = nullptr;
+  if (lane < 2 * P.S) {
+    const TensorArgs& A = issue_q ? P.q : P.k;
+    if (A.d != 0) {
+      my_bytes = (uint32_t)A.w * 2u;
+      my_src = reinterpret_cast<const unsigned char*>(A.x[is]);
+      my_dst = issue_q ? (uint32_t)is * (uint32_t)wa.q_slice_stride
+                       : (uint32_t)wa.k_base + (uint32_t)is * (uint32_t)wa.k_slice_stride;
+    }
+  }
+  const uint32_t row_bytes = ((uint32_t)P.q.d + (uint32_t)P.k.d) * 2u;
+  const uint64_t policy = ptx::policy_evict_first();
+  auto arm = [&](long long t) {  // whole warp
+    if (lane == 0) ptx::mbar_arrive_expect_tx(bar, row_bytes);
+    __syncwarp();
+    if (my_bytes) ptx::bulk_load(stage_u32 + my_dst, my_src + (unsigned long long)t * my_bytes, my_bytes, bar, policy);
+  };
+
+  const int cta_warps = blockDim.x >> 5;
+  const long long first = (long long)blockIdx.x * cta_warps + warp;
+  const long long step = (long long)gridDim.x * cta_warps;
+  __syncwarp();  // the warp's mbarrier is initialised (lane 0 did it above)
+  if (first < P.T) arm(first);
+
+  // gamma, once per CTA (the first rows are already on their way): slot j of lane `lane`,
+  // the slots dealt round-robin to the CTA's warps
+  {
+    const uint4* gq = reinterpret_cast<const uint4*>(P.q.gamma[ss]) + l;
+    const uint4* gk = reinterpret_cast<const uint4*>(P.k.gamma[ss]) + l;
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    for (int j = warp; j < L; j += cta_warps) {
+      uint4 v = zero;
+      if (j < nvq) v = __ldg(gq + (size_t)j * g);
+      else if (j >= wa.nq4 && j - wa.nq4 < nvk) v = __ldg(gk + (size_t)(j - wa.nq4) * g);
+      gsm[j][lane] = v;
+    }
+  }
+  __syncthreads();  // the only block-level barrier
+
+
+  // ---- loop-invariant per-lane offsets ------------------------------------------------------------
+  // inside a stage: chunk l of the lane's Q slice / K slice
+  const uint32_t sq0 = stage_u32 + (uint32_t)ss * (uint32_t)wa.q_slice_stride + (uint32_t)l * 16u;
+  const uint32_t sk0 = stage_u32 + (uint32_t)wa.k_base + (uint32_t)ss * (uint32_t)wa.k_slice_stride + (uint32_t)l * 16u;
+  const uint32_t szero = stage_u32 + (uint32_t)wa.zero_off;
+  const uint32_t sstride = (uint32_t)g * 16u;
+  unsigned char* yq = reinterpret_cast<unsigned char*>(P.q.y[ss]) + (size_t)l * 16u;
+  unsigned char* yk = reinterpret_cast<unsigned char*>(P.k.y[ss]) + (size_t)l * 16u;
+  const unsigned long long q_row = (unsigned long long)P.q.w * 2ull, k_row = (unsigned long long)P.k.w * 2ull;
+
+  uint32_t phase = 0;
+  for (long long t = first; t < P.T; t += step) {
+    if (!ptx::mbar_wait_bounded(bar, phase)) {
+      atomicCAS(wa.error_word, 0, 2);  // 2 = a warp's stage never arrived
+      return;
+    }
+    phase ^= 1u;
+    // ---- drain the stage into registers --------------------------------------------------------
+    uint4 v[L];
+#pragma unroll
+    for (int jb = 0; jb < L; jb += 4) {
+      if (jb >= n_slots) break;
+      const bool kpart = jb >= wa.nq4;  // uniform: a block of 4 slots is all Q or all K
+      const uint32_t base = kpart ? sk0 + (uint32_t)(jb - wa.nq4) * sstride : sq0 + (uint32_t)jb * sstride;
+      const int nv = kpart ? nvk - (jb - wa.nq4) : nvq - jb;  // slots of this block the lane has
+#pragma unroll
+      for (int i = 0; i < 4; ++i) v[jb + i] = ptx::lds128((EXACT || i < nv) ? base + (uint32_t)i * sstride : szero);
+    }
+    // ---- Phase A: sums of squares of the lane's Q chunks and K chunks ---------------------------------
+    float2 aq = make_float2(0.f, 0.f), ak = make_float2(0.f, 0.f);
+#pragma unroll
+    for (int jb = 0; jb < L; jb += 4) {
+      if (jb >= n_slots) break;
+      // four independent chains (one per chunk slot), two accumulators each
+      float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, c4 = 0.f, c5 = 0.f, c6 = 0.f, c7 = 0.f;
+      fma_bf16x2_sq(v[jb].x, c0, c1);
+      fma_bf16x2_sq(v[jb + 1].x, c2, c3);
+      fma_bf16x2_sq(v[jb + 2].x, c4, c5);
+      fma_bf16x2_sq(v[jb + 3].x, c6, c7);
+      fma_bf16x2_sq(v[jb].y, c0, c1);
+      fma_bf16x2_sq(v[jb + 1].y, c2, c3);
+      fma_bf16x2_sq(v[jb + 2].y, c4, c5);
+      fma_bf16x2_sq(v[jb + 3].y, c6, c7);
+      fma_bf16x2_sq(v[jb].z, c0, c1);
+      fma_bf16x2_sq(v[jb + 1].z, c2, c3);
+      fma_bf16x2_sq(v[jb + 2].z, c4, c5);
+      fma_bf16x2_sq(v[jb + 3].z, c6, c7);
+      fma_bf16x2_sq(v[jb].w, c0, c1);
+      fma_bf16x2_sq(v[jb + 1].w, c2, c3);
+      fma_bf16x2_sq(v[jb + 2].w, c4, c5);
+      fma_bf16x2_sq(v[jb + 3].w, c6, c7);
+      const float2 b = __fadd2_rn(__fadd2_rn(make_float2(c0, c1), make_float2(c2, c3)),
+                                  __fadd2_rn(make_float2(c4, c5), make_float2(c6, c7)));
+      if (jb >= wa.nq4) ak = __fadd2_rn(ak, b);
+      else aq = __fadd2_rn(aq, b);
+    }
+    float pq = aq.x + aq.y, pk = ak.x + ak.y;
+    if (g > 16) { pq += __shfl_xor_sync(0xffffffffu, pq, 16); pk += __shfl_xor_sync(0xffffffffu, pk, 16); }
+    if (g > 8) { pq += __shfl_xor_sync(0xffffffffu, pq, 8); pk += __shfl_xor_sync(0xffffffffu, pk, 8); }
+    if (g > 4) { pq += __shfl_xor_sync(0xffffffffu, pq, 4); pk += __shfl_xor_sync(0xffffffffu, pk, 4); }
+    if (g > 2) { pq += __shfl_xor_sync(0xffffffffu, pq, 2); pk += __shfl_xor_sync(0xffffffffu, pk, 2); }
+    if (g > 1) { pq += __shfl_xor_sync(0xffffffffu, pq, 1); pk += __shfl_xor_sync(0xffffffffu, pk, 1); }
+    // ---- the slices' scalars in ascending slice order -------------------------------------------------
+    float totq = pq, totk = pk;
+    if (P.S > 1) {
+      totq = 0.f;
+      totk = 0.f;
+      for (int s2 = 0; s2 < P.S; ++s2) {
+        totq += __shfl_sync(0xffffffffu, pq, s2 << wa.log_g);
+        totk += __shfl_sync(0xffffffffu, pk, s2 << wa.log_g);
+      }
+    } else {
+      totq = __shfl_sync(0xffffffffu, pq, 0);  // also the point where every lane has consumed the stage
+      totk = __shfl_sync(0xffffffffu, pk, 0);
+    }
+    // every lane's chunks are in registers and have been used: refill the stage with the next token
+    if (t + step < P.T) arm(t + step);
+
+    const float rq = rsqrtf(fmaf(totq, P.q.inv_d, P.eps));
+    const float rk = rsqrtf(fmaf(totk, P.k.inv_d, P.eps));
+    if (lane == 0) {
+      if (P.q.rstd != nullptr) P.q.rstd[t] = rq;
+      if (P.k.rstd != nullptr) P.k.rstd[t] = rk;
+    }
+    if (active && l == 0) {
+      if (P.q.partials != nullptr) P.q.partials[(long long)s * P.T + t] = pq;
+      if (P.k.partials != nullptr) P.k.partials[(long long)s * P.T + t] = pk;
+    }
+    // ---- Phases B/C: (x * gamma) * RMS^-1, the one write ------------------------------------------------
+    unsigned char* dq_ = yq + (unsigned long long)t * q_row;
+    unsigned char* dk_ = yk + (unsigned long long)t * k_row;
+#pragma unroll
+    for (int jb = 0; jb < L; jb += 4) {
+      if (jb >= n_slots) break;
+      const bool kpart = jb >= wa.nq4;
+      const float r = kpart ? rk : rq;
+      const float2 r2 = make_float2(r, r);
+      unsigned char* dst = kpart ? dk_ + (size_t)(jb - wa.nq4) * sstride : dq_ + (size_t)jb * sstride;
+      const int nv = kpart ? (EXACT ? wa.nk : nvk) - (jb - wa.nq4) : (EXACT ? wa.nq : nvq) - jb;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint4 o = scale_chunk_mixed(v[jb + i], gsm[jb + i][lane], r2);
+        if (i < nv) st_stream(reinterpret_cast<uint4*>(dst + (size_t)i * sstride), o);
+      }
+    }
+  }
+}
+
+using WarpKernel = void (*)(const Params, const WarpArgs);
+WarpKernel warp_kernel_for(int l, bool exact);  // nullptr outside the instantiated set
+int warp_round_up_l(int n);                      // next instantiated L >= n, or -1
+
+}  // namespace qknorm

@@ -140,7 +140,7 @@ def small_parity_shapes() -> List[Workload]:
         ("s_24", 5, 24, 8, (1,)),
         ("s_unaligned", 7, 1001, 77, (1, 7)),
         ("s_149", 149, 5120, 1024, (1, 8)),
-        ("s_1025", 1025, 640, 128, (1, 5)),
+        ("s_1025", 1025, 640, 128, (1, 4)),
         ("s_8200", 33, 8200, 8200, (1, 5)),
         ("s_wide", 9, 16384, 2048, (1, 16)),
         ("s_max", 2, 65536, 8, (1,)),
@@ -148,6 +148,11 @@ def small_parity_shapes() -> List[Workload]:
         ("s_mha4", 257, 5120, 5120, (4,)),
         ("s_konly", 17, 0, 1024, (1, 4)),
         ("s_qonly", 17, 2048, 0, (1, 4)),
+        ("s_prefill_gqa", 1500, 5120, 1024, (8, 1)),     # warp-per-token kernel, several rows per warp
+        ("s_prefill_odd", 777, 1000, 136, (1,)),         # warp-per-token kernel, lanes with ragged chunk counts
+        ("s_prefill_s3", 650, 1536, 768, (3,)),          # shard count that leaves lanes idle
+        ("s_prefill_konly", 700, 0, 1024, (2,)),
+        ("s_prefill_wide", 600, 16384, 4096, (1, 4)),    # rows too wide for one warp: the CTA-per-token TMA ring
     ]
     out = []
     for i, (name, t, dq, dk, sh) in enumerate(shapes):

@@ -119,11 +119,18 @@ def test_unaligned_buffers_take_the_general_kernel(libqknorm, skew):
         check_against_oracle(w, S, res)
 
 
-def test_vector_kernel_is_the_one_that_runs_on_aligned_shapes(libqknorm):
-    for name in ("s_149", "s_gqa8", "s_t1"):
-        w = next(x for x in SMALL if x.name == name)
-        res = run_case(w, w.shards[0])
-        assert res["variant"] == "rows", (name, res["variant"])
+@pytest.mark.parametrize("name,S,variant", [
+    ("s_t1", 1, "rows"), ("s_149", 8, "rows"), ("s_gqa8", 8, "rows"),          # few tokens: register-resident rows
+    ("s_prefill_gqa", 8, "warp"), ("s_prefill_gqa", 1, "warp"), ("s_prefill_odd", 1, "warp"),
+    ("s_prefill_s3", 3, "warp"), ("s_prefill_konly", 2, "warp"), ("s_1025", 4, "warp"),
+    ("s_prefill_wide", 1, "ring"), ("s_prefill_wide", 4, "ring"),
+    ("s_unaligned", 7, "general"), ("s_max", 1, "general"),
+])
+def test_every_kernel_variant_is_exercised(libqknorm, name, S, variant):
+    w = next(x for x in SMALL if x.name == name)
+    res = run_case(w, S)
+    assert res["variant"] == variant, (name, S, res["variant"])
+    check_against_oracle(w, S, res)
 
 
 def test_results_are_bitwise_reproducible(libqknorm):

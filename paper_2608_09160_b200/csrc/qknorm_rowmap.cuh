@@ -32,8 +32,8 @@ namespace qknorm {
 
 // Largest CTA the kernels with N chunks per thread are compiled for, and how
 // many such CTAs the register budget is shaped for.
-__host__ __device__ constexpr int max_threads_for(int n) { return n <= 2 ? 1024 : (n <= 4 ? 384 : 256); }
-__host__ __device__ constexpr int min_blocks_for(int n) { return n <= 2 ? 1 : (n <= 6 ? 2 : 1); }
+__host__ __device__ constexpr int max_threads_for(int n) { return n <= 2 ? 1024 : 512; }
+__host__ __device__ constexpr int min_blocks_for(int) { return 1; }
 
 struct LaneMap {
   bool active;        // this thread serves a slice

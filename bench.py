@@ -50,9 +50,12 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per launch of the dominant kernel measured by ncu
-# (dram__bytes_read.sum + dram__bytes_write.sum); the capture each figure comes
-# from is summarised under profiles/.  None = not captured.
-NCU_DRAM_TRAFFIC_BYTES = {}
+# (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
+# C5/S8: captured on 16384 of the 65536 tokens (302.05 MB read + 246.77 MB
+# written per launch, profiles/warp_kernel_C5_16k_tokens_full_set.md) and scaled
+# by the tokens processed (x4).  Reads scale exactly; the writes fall short of
+# the algorithmic bytes by the lines still dirty in L2 when the kernel ends.
+NCU_DRAM_TRAFFIC_BYTES = {"C5/S8": 4 * (302_049_152 + 246_769_920)}
 
 
 def log(*a):
@@ -306,6 +309,19 @@ def cpu_baseline(w: W.Workload, target_cpu_seconds: float = 16.0):
             "seconds": round(dt, 3)}
 
 
+def config_of(w: W.Workload, S: int, world: int, variant=None):
+    """The `config` object of the JSON line (the same for both arms)."""
+    cfg = {"workload": f"{w.name}: {w.note}", "tokens": w.tokens, "dq": w.dq, "dk": w.dk, "num_shards": S,
+           "in_place": w.in_place, "storage": "bf16", "eps": w.eps,
+           "bytes_per_step_per_gpu": w.algorithmic_bytes,
+           "parallelism": f"token-range x{world}, no collective",
+           "l2": "inputs larger than L2 (no flush needed)" if w.algorithmic_bytes > 300e6
+                 else "working set fits in L2 (L2-warm number)"}
+    if variant is not None:
+        cfg["kernel_variant"] = variant
+    return cfg
+
+
 def run_reference(args):
     """--impl reference: the oracle as it stands, on host cores, rank 0 only."""
     rank = int(os.environ.get("RANK", "0"))
@@ -313,6 +329,9 @@ def run_reference(args):
         return 0
     import oracle
     w = W.WORKLOADS[args.workload]
+    if args.tokens:
+        w = W.scaled(w, args.tokens)
+    S = args.shards or w.shards[0]
     cores = min(os.cpu_count() or 1, oracle.max_threads())
     ws, bits = oracle_sample_inputs(w, 256)
     run_oracle_once(bits, w.eps, cores)
@@ -332,7 +351,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": round(gbs, 4), "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(total / args.steps * 1e3, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "tokens": w.tokens, "dq": w.dq, "dk": w.dk, "sample_tokens": n},
+        "config": {**config_of(w, S, 1), "sample_tokens_per_step": n},
         "cpu_baseline": {"value": round(gbs, 4), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": round(gbs, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -454,12 +473,7 @@ def main():
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{w.name}: {w.note}", "tokens": w.tokens, "dq": w.dq, "dk": w.dk,
-                   "num_shards": S, "in_place": w.in_place, "storage": "bf16", "eps": w.eps,
-                   "bytes_per_step_per_gpu": w.algorithmic_bytes, "parallelism": f"token-range x{world}, no collective",
-                   "l2": "inputs larger than L2 (no flush needed)" if w.algorithmic_bytes > 300e6
-                         else "working set fits in L2 (L2-warm number)",
-                   "kernel_variant": variant},
+        "config": config_of(w, S, world, variant),
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": int(launches),

@@ -16,34 +16,6 @@ __device__ __forceinline__ uint32_t bf_pack(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&r);
 }
 
-// Sum of squares of the 8 values of a 16-byte chunk, added to acc (fp32 FMA chain).
-__device__ __forceinline__ float chunk_sumsq(const uint4& v, float acc) {
-  acc = fmaf(bf_lo(v.x), bf_lo(v.x), acc);
-  acc = fmaf(bf_hi(v.x), bf_hi(v.x), acc);
-  acc = fmaf(bf_lo(v.y), bf_lo(v.y), acc);
-  acc = fmaf(bf_hi(v.y), bf_hi(v.y), acc);
-  acc = fmaf(bf_lo(v.z), bf_lo(v.z), acc);
-  acc = fmaf(bf_hi(v.z), bf_hi(v.z), acc);
-  acc = fmaf(bf_lo(v.w), bf_lo(v.w), acc);
-  acc = fmaf(bf_hi(v.w), bf_hi(v.w), acc);
-  return acc;
-}
-
-// (x * gamma) * rstd on one packed word (Algorithm 1: the weight multiply of
-// Phase B, then the scaling of Phase C), rounded once.
-__device__ __forceinline__ uint32_t scale_word(uint32_t x, uint32_t g, float rstd) {
-  return bf_pack((bf_lo(x) * bf_lo(g)) * rstd, (bf_hi(x) * bf_hi(g)) * rstd);
-}
-
-__device__ __forceinline__ uint4 scale_chunk(const uint4& x, const uint4& g, float rstd) {
-  uint4 o;
-  o.x = scale_word(x.x, g.x, rstd);
-  o.y = scale_word(x.y, g.y, rstd);
-  o.z = scale_word(x.z, g.z, rstd);
-  o.w = scale_word(x.w, g.w, rstd);
-  return o;
-}
-
 // Mixed-precision FMA of sm_100 (PTX fma.rn.f32.bf16): d = a*b + c with a, b the
 // bf16 halves of packed words and c, d fp32.  The product of two bf16 values is
 // exact in fp32, so this rounds exactly like widening first and using an fp32

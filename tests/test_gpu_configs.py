@@ -66,3 +66,30 @@ def test_full_size_workload(libqknorm, name, S):
         assert bool(torch.isfinite(y).all())
         bound = inp["gamma_" + nm].float().abs() * (d ** 0.5) * (1 + 2 ** -7)
         assert bool((y.abs() <= bound[None, :]).all())
+
+
+def test_rows_beyond_2_to_the_31_elements(libqknorm):
+    """Index arithmetic: a Q tensor of 2.3e9 elements (4.6 GB), so byte and element offsets of
+    the last rows do not fit in 32 bits.  The tensor is a 2048-token seeded block repeated along
+    the token axis, so every row has a known oracle row; rows near the end are compared."""
+    base = W.Workload("big_base", tokens=2048, dq=8192, dk=1024, shards=(8,), seed=21)
+    inp = W.make_inputs(base)
+    reps = 140                                   # 286720 tokens x 8192 = 2.35e9 elements
+    T = base.tokens * reps
+    S = 8
+    qs = [t.cuda().repeat(reps, 1) for t in W.shard_columns(inp["q"], S)]
+    ks = [t.cuda().repeat(reps, 1) for t in W.shard_columns(inp["k"], S)]
+    gqs = [t.cuda() for t in W.shard_columns(inp["gamma_q"], S)]
+    gks = [t.cuda() for t in W.shard_columns(inp["gamma_k"], S)]
+    assert sum(t.numel() for t in qs) > 2 ** 31
+    binding.qknorm_fwd_sharded(qs, ks, gqs, gks, base.eps, qs, ks)      # in place
+    torch.cuda.synchronize()
+    ref = H.oracle_unsharded(inp, base.eps, nthreads=NTHREADS)
+    for lo in (0, T // 2 - 1024, T - 2048):                              # first, middle, last block of rows
+        got_q = W.unshard_columns([t[lo:lo + 2048].cpu() for t in qs])
+        got_k = W.unshard_columns([t[lo:lo + 2048].cpu() for t in ks])
+        shift = lo % base.tokens
+        want_q = np.roll(ref["q"]["y"], -shift, axis=0)
+        want_k = np.roll(ref["k"]["y"], -shift, axis=0)
+        H.compare_output(W.bf16_bits(got_q), want_q, f"rows {lo}.. q")
+        H.compare_output(W.bf16_bits(got_k), want_k, f"rows {lo}.. k")

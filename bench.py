@@ -147,12 +147,11 @@ class DeviceCase:
     """Device (and optionally pinned host) buffers of one workload at one shard
     count, plus the closure that makes the one C-ABI call."""
 
-    def __init__(self, w: W.Workload, S: int, seed_offset: int = 0, host: bool = False):
+    def __init__(self, w: W.Workload, S: int, rank: int = 0, host: bool = False):
         from paper_2608_09160_b200 import binding
         self.binding = binding
         self.w, self.S = w, S
-        ww = W.Workload(**{**w.__dict__, "seed": w.seed + seed_offset})
-        inp = W.make_inputs(ww)
+        inp = W.make_inputs(rank_workload(w, rank))
         self.host_in = None
         if S == 1:
             host_parts = {"q": [inp["q"]], "k": [inp["k"]], "gq": [inp["gamma_q"]], "gk": [inp["gamma_k"]]}
@@ -356,6 +355,26 @@ def cpu_baseline(w: W.Workload, target_cpu_seconds: float = 16.0):
             "seconds": round(dt, 3)}
 
 
+def rank_workload(w: W.Workload, rank: int) -> W.Workload:
+    """The path shards by token range with no exchange: rank r normalises its own tokens.
+    Weak scaling: every rank gets the workload's shape with its own seed (its own tokens)."""
+    return W.Workload(**{**w.__dict__, "seed": w.seed + 1000 * rank})
+
+
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Job time = the slowest rank's device time (all_reduce MAX); identity on one rank."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(bytes_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job GB/s: the bytes all ranks processed in the time the slowest one took."""
+    return world * bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 def config_of(w: W.Workload, S: int, world: int, variant=None):
     """The `config` object of the JSON line (the same for both arms)."""
     cfg = {"workload": f"{w.name}: {w.note}", "tokens": w.tokens, "dq": w.dq, "dk": w.dk, "num_shards": S,
@@ -459,7 +478,7 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    case = DeviceCase(w, S, seed_offset=1000 * rank, host=not args.no_e2e)
+    case = DeviceCase(w, S, rank=rank, host=not args.no_e2e)
 
     # ---- device-resident timing -----------------------------------------------------------
     for _ in range(args.warmup):
@@ -474,12 +493,9 @@ def main():
     total_ms = time_region(case.call, args.steps)            # the K timed steps, back to back
     barrier()
     launches = binding.launch_count() - n0
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, "cuda")
     ms_per_step = total_ms / args.steps
-    value = world * case.bytes / (ms_per_step * 1e-3) / 1e9
+    value = job_value(case.bytes, world, ms_per_step)
     launch_ms = statistics.mean(per_call)
     achieved = case.bytes / (launch_ms * 1e-3) / 1e9
 
@@ -492,12 +508,9 @@ def main():
         barrier()
         e_ms = time_region(case.e2e_step, args.steps)
         barrier()
-        if dist is not None:
-            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = max_over_ranks(e_ms, dist, "cuda")
         h2d, d2h = case.e2e_bytes()
-        e2e = {"value": round(world * case.bytes / (e_ms / args.steps * 1e-3) / 1e9, 3), "unit": UNIT,
+        e2e = {"value": round(job_value(case.bytes, world, e_ms / args.steps), 3), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "ms_per_step": round(e_ms / args.steps, 3), "calls_per_step": e2e_chunks,
                "how": "pinned host buffers -> device -> C-ABI call -> pinned host buffers, in token chunks "

@@ -11,4 +11,7 @@ from .qknorm_oracle import (  # noqa: F401
     bf16_to_f64,
     f64_to_bf16,
     max_threads,
+    e4m3_to_f64,
+    f64_to_e4m3,
+    rmsnorm_e4m3,
 )

@@ -181,6 +181,115 @@ int qko_rmsnorm_sharded(const uint16_t* const* x_shards, const uint16_t* const* 
     return 0;
 }
 
+/* ---- FP8-E4M3 activations (Section IV-C: "BF16 and FP8-E4M3 activations", FP32 accumulation) ----
+ *
+ * The same definition (Eq. 1) with the activations stored as FP8 E4M3 (1 sign, 4
+ * exponent bits with bias 7, 3 mantissa bits; no infinities, S.1111.111 is NaN,
+ * largest finite value 448).  gamma stays bf16.  The output is rounded from fp64
+ * to E4M3 in ONE step, to nearest even, and values beyond the largest finite
+ * value saturate to +-448 (the paper does not say; this is the conversion the
+ * hardware offers, cvt.rn.satfinite). */
+
+double qko_e4m3_to_f64(uint8_t b) {
+    const int sign = b >> 7, ex = (b >> 3) & 15, man = b & 7;
+    double v;
+    if (ex == 15 && man == 7) return sign ? -NAN : NAN;
+    if (ex == 0) v = ldexp((double)man, -9);              /* subnormal: man/8 * 2^-6 */
+    else v = ldexp(1.0 + (double)man / 8.0, ex - 7);
+    return sign ? -v : v;
+}
+
+uint8_t qko_f64_to_e4m3(double v) {
+    const uint8_t sign = signbit(v) ? 0x80u : 0x00u;
+    if (isnan(v)) return (uint8_t)(sign | 0x7Fu);
+    double a = fabs(v);
+    if (a == 0.0) return sign;
+    if (isinf(a)) return (uint8_t)(sign | 0x7Eu);         /* saturate */
+    int ex;
+    (void)frexp(a, &ex);
+    int e = ex - 1;                                        /* floor(log2 a) */
+    if (e < -6) e = -6;                                    /* subnormals share the smallest normal's unit */
+    const double unit = ldexp(1.0, e - 3);                 /* 4 significant bits */
+    double r = nearbyint(a / unit) * unit;                 /* nearest, ties to even */
+    if (r > 448.0) r = 448.0;                              /* saturate to the largest finite value */
+    if (r == 0.0) return sign;
+    int rex;
+    const double m = frexp(r, &rex);                       /* r = m * 2^rex, 0.5 <= m < 1 */
+    int re = rex - 1;
+    uint8_t bits;
+    if (re < -6) {                                         /* subnormal: r = man * 2^-9 */
+        bits = (uint8_t)(int)(r * 512.0);
+    } else {
+        const int man = (int)((m * 2.0 - 1.0) * 8.0);      /* exact: r has at most 4 significant bits */
+        bits = (uint8_t)(((re + 7) << 3) | man);
+    }
+    return (uint8_t)(sign | bits);
+}
+
+static void rmsnorm_row_e4m3(const uint8_t* x, const uint16_t* gamma, int64_t H, double eps,
+                             uint8_t* y, double* y64, double* acc_out, double* rstd_out) {
+    double acc = 0.0;
+    for (int64_t j = 0; j < H; ++j) {
+        double v = qko_e4m3_to_f64(x[j]);
+        acc += v * v;
+    }
+    double r = 1.0 / sqrt(acc / (double)H + eps);
+    for (int64_t j = 0; j < H; ++j) {
+        double o = qko_e4m3_to_f64(x[j]) * r * qko_bf16_to_f64(gamma[j]);
+        if (y64) y64[j] = o;
+        if (y) y[j] = qko_f64_to_e4m3(o);
+    }
+    if (acc_out) *acc_out = acc;
+    if (rstd_out) *rstd_out = r;
+}
+
+/* x_shards[s]: [T][H/S] E4M3 bytes; gamma_shards[s]: [H/S] bf16.  S == 1 is the unsharded
+ * form.  Same conventions as qko_rmsnorm_sharded (gather, Eq. 1 with the full width, cut back). */
+int qko_rmsnorm_sharded_e4m3(const uint8_t* const* x_shards, const uint16_t* const* gamma_shards,
+                             int S, int64_t T, int64_t H, float eps, uint8_t* const* y_shards,
+                             double* y64, double* partials, double* acc, double* rstd, int nthreads) {
+    if (S < 1 || T < 0 || H < 0 || (H % S) != 0) return -1;
+    if (T == 0 || H == 0) return 0;
+    if (!x_shards || !gamma_shards) return -1;
+    const int64_t w = H / S;
+    const double e = (double)eps;
+    uint16_t* gfull = (uint16_t*)malloc((size_t)H * sizeof(uint16_t));
+    if (!gfull) return -1;
+    for (int s = 0; s < S; ++s) memcpy(gfull + s * w, gamma_shards[s], (size_t)w * sizeof(uint16_t));
+    int nt = 1;
+#ifdef _OPENMP
+    if (nthreads > 1) nt = nthreads;
+#pragma omp parallel for num_threads(nt) schedule(static)
+#else
+    (void)nthreads;
+#endif
+    for (int64_t t = 0; t < T; ++t) {
+        uint8_t* row = (uint8_t*)malloc((size_t)H);
+        uint8_t* out = (uint8_t*)malloc((size_t)H);
+        for (int s = 0; s < S; ++s) memcpy(row + s * w, x_shards[s] + t * w, (size_t)w);
+        if (partials) {
+            for (int s = 0; s < S; ++s) {
+                double p = 0.0;
+                for (int64_t j = 0; j < w; ++j) {
+                    double v = qko_e4m3_to_f64(x_shards[s][t * w + j]);
+                    p += v * v;
+                }
+                partials[(int64_t)s * T + t] = p;
+            }
+        }
+        rmsnorm_row_e4m3(row, gfull, H, e, out, y64 ? y64 + t * H : NULL, acc ? acc + t : NULL,
+                         rstd ? rstd + t : NULL);
+        if (y_shards) {
+            for (int s = 0; s < S; ++s)
+                if (y_shards[s]) memcpy(y_shards[s] + t * w, out + s * w, (size_t)w);
+        }
+        free(row);
+        free(out);
+    }
+    free(gfull);
+    return 0;
+}
+
 /* Threads the OpenMP build will actually use when asked for n. */
 int qko_max_threads(void) {
 #ifdef _OPENMP

@@ -19,6 +19,7 @@ _lib = None
 
 _u16p = ctypes.POINTER(ctypes.c_uint16)
 _f64p = ctypes.POINTER(ctypes.c_double)
+_u8p = ctypes.POINTER(ctypes.c_uint8)
 
 
 def build(force: bool = False) -> str:
@@ -50,6 +51,14 @@ def _load():
         lib.qko_rmsnorm_sharded.argtypes = [pp, pp, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
                                             ctypes.c_float, pp, _f64p, _f64p, _f64p, ctypes.c_int]
         lib.qko_rmsnorm_sharded.restype = ctypes.c_int
+        lib.qko_e4m3_to_f64.argtypes = [ctypes.c_uint8]
+        lib.qko_e4m3_to_f64.restype = ctypes.c_double
+        lib.qko_f64_to_e4m3.argtypes = [ctypes.c_double]
+        lib.qko_f64_to_e4m3.restype = ctypes.c_uint8
+        p8 = ctypes.POINTER(_u8p)
+        lib.qko_rmsnorm_sharded_e4m3.argtypes = [p8, pp, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
+                                                 ctypes.c_float, p8, _f64p, _f64p, _f64p, _f64p, ctypes.c_int]
+        lib.qko_rmsnorm_sharded_e4m3.restype = ctypes.c_int
         lib.qko_max_threads.argtypes = []
         lib.qko_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -143,3 +152,56 @@ def rmsnorm_sharded(x_shards: Sequence[np.ndarray], gamma_shards: Sequence[np.nd
     if rc != 0:
         raise RuntimeError(f"qko_rmsnorm_sharded failed ({rc})")
     return {"y": ys, "partials": partials, "acc": acc, "rstd": rstd}
+
+
+def e4m3_to_f64(bits) -> np.ndarray:
+    lib = _load()
+    b = np.asarray(bits, dtype=np.uint8)
+    out = np.empty(b.shape, dtype=np.float64)
+    fo, fb = out.reshape(-1), b.reshape(-1)
+    for i in range(fb.size):
+        fo[i] = lib.qko_e4m3_to_f64(int(fb[i]))
+    return out
+
+
+def f64_to_e4m3(vals) -> np.ndarray:
+    lib = _load()
+    v = np.asarray(vals, dtype=np.float64)
+    out = np.empty(v.shape, dtype=np.uint8)
+    fo, fv = out.reshape(-1), v.reshape(-1)
+    for i in range(fv.size):
+        fo[i] = lib.qko_f64_to_e4m3(float(fv[i]))
+    return out
+
+
+def rmsnorm_e4m3(x_shards: Sequence[np.ndarray], gamma_shards: Sequence[np.ndarray], eps: float, *,
+                 want_y64: bool = False, nthreads: int = 1):
+    """Eq. 1 with FP8-E4M3 activations (uint8 bit patterns) and bf16 gamma (uint16 bit
+    patterns), given as S column slices (S = 1: unsharded).  Returns y (list of uint8
+    [T,w]), partials (fp64 [S,T]), acc, rstd (fp64 [T]) and, if asked, y64 ([T,H])."""
+    lib = _load()
+    S = len(x_shards)
+    if S < 1 or len(gamma_shards) != S:
+        raise ValueError("need S >= 1 shards and as many gamma slices")
+    xs = [np.ascontiguousarray(a) for a in x_shards]
+    gs = [_u16(a) for a in gamma_shards]
+    T, w = xs[0].shape
+    for a, g in zip(xs, gs):
+        if a.dtype != np.uint8 or a.shape != (T, w) or g.shape != (w,):
+            raise ValueError("all shards must be uint8 [T,w] with gamma uint16 [w]")
+    ys = [np.empty((T, w), dtype=np.uint8) for _ in range(S)]
+    y64 = np.empty((T, w * S), dtype=np.float64) if want_y64 else None
+    partials = np.empty((S, T), dtype=np.float64)
+    acc = np.empty((T,), dtype=np.float64)
+    rstd = np.empty((T,), dtype=np.float64)
+    xa = (_u8p * S)(*[_ptr(a, _u8p) for a in xs])
+    ga = (_u16p * S)(*[_ptr(a, _u16p) for a in gs])
+    ya = (_u8p * S)(*[_ptr(a, _u8p) for a in ys])
+    rc = lib.qko_rmsnorm_sharded_e4m3(xa, ga, S, T, w * S, float(eps), ya, _ptr(y64, _f64p),
+                                      _ptr(partials, _f64p), _ptr(acc, _f64p), _ptr(rstd, _f64p), int(nthreads))
+    if rc != 0:
+        raise RuntimeError(f"qko_rmsnorm_sharded_e4m3 failed ({rc})")
+    res = {"y": ys, "partials": partials, "acc": acc, "rstd": rstd}
+    if want_y64:
+        res["y64"] = y64
+    return res

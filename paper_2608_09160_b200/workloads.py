@@ -98,6 +98,37 @@ def make_inputs(w: Workload) -> Dict[str, torch.Tensor]:
     }
 
 
+E4M3_MAX = 448.0
+
+
+def make_inputs_e4m3(w: Workload) -> Dict[str, torch.Tensor]:
+    """The same draws as make_inputs with the activations rounded ONCE from fp32 to FP8-E4M3
+    (torch.float8_e4m3fn; fp32 values are clamped to the finite range first).  gamma stays bf16."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(int(w.seed))
+    q = torch.empty((w.tokens, w.dq), dtype=torch.float32).normal_(0.0, w.sigma, generator=gen)
+    k = torch.empty((w.tokens, w.dk), dtype=torch.float32).normal_(0.0, w.sigma, generator=gen)
+    gq = torch.empty((w.dq,), dtype=torch.float32).uniform_(0.5, 1.5, generator=gen)
+    gk = torch.empty((w.dk,), dtype=torch.float32).uniform_(0.5, 1.5, generator=gen)
+    if w.outlier_frac > 0.0:
+        cq = _outlier_channels(w.dq, w.outlier_frac, gen)
+        ck = _outlier_channels(w.dk, w.outlier_frac, gen)
+        q[:, cq] *= w.outlier_scale
+        k[:, ck] *= w.outlier_scale
+    return {
+        "q": q.clamp_(-E4M3_MAX, E4M3_MAX).to(torch.float8_e4m3fn),
+        "k": k.clamp_(-E4M3_MAX, E4M3_MAX).to(torch.float8_e4m3fn),
+        "gamma_q": gq.to(torch.bfloat16),
+        "gamma_k": gk.to(torch.bfloat16),
+    }
+
+
+def e4m3_bits(x: torch.Tensor):
+    """Raw bit patterns of a CPU float8_e4m3fn tensor as a numpy uint8 array (a view)."""
+    assert x.dtype == torch.float8_e4m3fn and x.device.type == "cpu"
+    return x.contiguous().view(torch.uint8).numpy()
+
+
 def shard_columns(x: torch.Tensor, num_shards: int) -> List[torch.Tensor]:
     """Equal contiguous column slices, slice s = columns [s*w, (s+1)*w), each in
     its own contiguous buffer (the layout a column-parallel projection leaves on

@@ -31,3 +31,24 @@ def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
     """Widening through numpy (used to express expected values, not to compute the method)."""
     b = np.asarray(bits, dtype=np.uint16)
     return (b.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def e4m3_ordinal(bits: np.ndarray) -> np.ndarray:
+    """Monotone integer order of FP8-E4M3 bit patterns (+0 and -0 both 0)."""
+    b = np.asarray(bits, dtype=np.uint8).astype(np.int32)
+    mag = b & 0x7F
+    return np.where((b & 0x80) != 0, -mag, mag)
+
+
+def e4m3_isnan(bits: np.ndarray) -> np.ndarray:
+    return (np.asarray(bits, dtype=np.uint8) & 0x7F) == 0x7F
+
+
+def e4m3_ordinal_distance(a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
+    a = np.asarray(a_bits, dtype=np.uint8)
+    b = np.asarray(b_bits, dtype=np.uint8)
+    d = np.abs(e4m3_ordinal(a) - e4m3_ordinal(b))
+    na, nb = e4m3_isnan(a), e4m3_isnan(b)
+    d = np.where(na & nb, 0, d)
+    d = np.where(na ^ nb, 1 << 20, d)
+    return d

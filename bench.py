@@ -147,11 +147,12 @@ class DeviceCase:
     """Device (and optionally pinned host) buffers of one workload at one shard
     count, plus the closure that makes the one C-ABI call."""
 
-    def __init__(self, w: W.Workload, S: int, rank: int = 0, host: bool = False):
+    def __init__(self, w: W.Workload, S: int, rank: int = 0, host: bool = False, io: str = "bf16"):
         from paper_2608_09160_b200 import binding
         self.binding = binding
-        self.w, self.S = w, S
-        inp = W.make_inputs(rank_workload(w, rank))
+        self.w, self.S, self.io = w, S, io
+        make = W.make_inputs if io == "bf16" else W.make_inputs_e4m3
+        inp = make(rank_workload(w, rank))
         self.host_in = None
         if S == 1:
             host_parts = {"q": [inp["q"]], "k": [inp["k"]], "gq": [inp["gamma_q"]], "gk": [inp["gamma_k"]]}
@@ -169,14 +170,18 @@ class DeviceCase:
             self.host_in = {k: [t.pin_memory() for t in host_parts[k]] for k in ("q", "k")}
             self.host_out = {"q": [torch.empty_like(t).pin_memory() for t in host_parts["q"]],
                              "k": [torch.empty_like(t).pin_memory() for t in host_parts["k"]]}
-        self.bytes = w.algorithmic_bytes
+        # every element read once and written once (1 or 2 bytes), every gamma (bf16) read once
+        eb = 2 if io == "bf16" else 1
+        self.bytes = 2 * w.tokens * (w.dq + w.dk) * eb + (w.dq + w.dk) * 2
+        self.fwd = binding.qknorm_fwd if io == "bf16" else binding.qknorm_fwd_e4m3
+        self.fwd_sharded = binding.qknorm_fwd_sharded if io == "bf16" else binding.qknorm_fwd_sharded_e4m3
 
     def call(self):
-        b, d = self.binding, self.dev
+        d = self.dev
         if self.S == 1:
-            b.qknorm_fwd(d["q"][0], d["k"][0], d["gq"][0], d["gk"][0], self.w.eps, self.out_q[0], self.out_k[0])
+            self.fwd(d["q"][0], d["k"][0], d["gq"][0], d["gk"][0], self.w.eps, self.out_q[0], self.out_k[0])
         else:
-            b.qknorm_fwd_sharded(d["q"], d["k"], d["gq"], d["gk"], self.w.eps, self.out_q, self.out_k)
+            self.fwd_sharded(d["q"], d["k"], d["gq"], d["gk"], self.w.eps, self.out_q, self.out_k)
 
     def prepare_e2e(self, nchunks: int = 8):
         """Cuts the step into token chunks so that the copy engines run in both directions
@@ -213,9 +218,9 @@ class DeviceCase:
                 ev_in = self.s_in.record_event()
             cur.wait_event(ev_in)
             if self.S == 1:
-                b.qknorm_fwd(c["q"][0], c["k"][0], d["gq"][0], d["gk"][0], self.w.eps, c["oq"][0], c["ok"][0])
+                self.fwd(c["q"][0], c["k"][0], d["gq"][0], d["gk"][0], self.w.eps, c["oq"][0], c["ok"][0])
             else:
-                b.qknorm_fwd_sharded(c["q"], c["k"], d["gq"], d["gk"], self.w.eps, c["oq"], c["ok"])
+                self.fwd_sharded(c["q"], c["k"], d["gq"], d["gk"], self.w.eps, c["oq"], c["ok"])
             self.s_out.wait_event(cur.record_event())
             with torch.cuda.stream(self.s_out):
                 for dst, src in c["d2h"]:
@@ -223,7 +228,7 @@ class DeviceCase:
         cur.wait_stream(self.s_out)
 
     def e2e_bytes(self):
-        n = sum(t.numel() * 2 for name in ("q", "k") for t in self.host_in[name])
+        n = sum(t.numel() * t.element_size() for name in ("q", "k") for t in self.host_in[name])
         return n, n
 
 
@@ -294,12 +299,16 @@ def config_table(steps: int, warmup: int, peak: float, skip: str):
     """us/call, GB/s and roofline fraction of every workload other than the headline one."""
     from paper_2608_09160_b200 import binding
     rows = {}
-    for name, w in W.WORKLOADS.items():
-        for S in w.shards:
-            key = f"{name}/S{S}"
+    todo = [(name, S, "bf16") for name, w in W.WORKLOADS.items() for S in w.shards]
+    # FP8-E4M3 activations (Section IV-C), the prefill workloads at their last shard count
+    todo += [(name, W.WORKLOADS[name].shards[-1], "e4m3") for name in ("C3", "C4", "C5")]
+    for name, S, io in todo:
+        w = W.WORKLOADS[name]
+        if True:
+            key = f"{name}/S{S}" + ("" if io == "bf16" else "/e4m3")
             if key == skip:
                 continue
-            case = DeviceCase(w, S)
+            case = DeviceCase(w, S, io=io)
             ts = time_calls(case.call, max(steps, 10), max(warmup, 3))
             med, mn = statistics.median(ts), min(ts)
             row = {"us_median": round(med * 1e3, 3), "us_min": round(mn * 1e3, 3),

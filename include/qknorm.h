@@ -111,6 +111,28 @@ int qknorm_fwd_sharded_ex(const void* const* q_shards, const void* const* k_shar
                           float* partials_q, float* partials_k, float* rstd_q, float* rstd_k,
                           void* stream);
 
+/*
+ * FP8-E4M3 activations (Section IV-C: "SwiftQK accumulates local squared sums and
+ * cross-GPU scalar reductions in FP32, even for BF16 and FP8-E4M3 activations").
+ * The same operation with q, k and the outputs stored as FP8 E4M3 (one byte per
+ * element: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities,
+ * S.1111.111 = NaN, largest finite value 448).  gamma stays bf16; all arithmetic is
+ * fp32; the result is rounded once to E4M3, to nearest even, saturating at +-448.
+ * Arguments as qknorm_fwd_ex / qknorm_fwd_sharded_ex (rstd_* and partials_* may be
+ * NULL).  Vectorised kernels need 16-byte aligned pointers and (shard) widths that
+ * are multiples of 16 elements; other shapes take the general kernel.
+ */
+int qknorm_fwd_e4m3(const void* q, const void* k, const void* gamma_q, const void* gamma_k,
+                    int64_t tokens, int32_t dq, int32_t dk, float eps,
+                    void* out_q, void* out_k, float* rstd_q, float* rstd_k, void* stream);
+
+int qknorm_fwd_sharded_e4m3(const void* const* q_shards, const void* const* k_shards,
+                            const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                            int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
+                            void* const* out_q_shards, void* const* out_k_shards,
+                            float* partials_q, float* partials_k, float* rstd_q, float* rstd_k,
+                            void* stream);
+
 /* Human-readable name of a qknorm_status (static storage, never NULL). */
 const char* qknorm_status_string(int status);
 

@@ -21,6 +21,8 @@ EXPORTS = (
     "qknorm_fwd_sharded",
     "qknorm_fwd_ex",
     "qknorm_fwd_sharded_ex",
+    "qknorm_fwd_e4m3",
+    "qknorm_fwd_sharded_e4m3",
     "qknorm_status_string",
     "qknorm_device_error_word",
     "qknorm_last_cuda_error",
@@ -69,6 +71,10 @@ def load() -> ctypes.CDLL:
     lib.qknorm_fwd_sharded_ex.argtypes = [_vpp, _vpp, _vpp, _vpp, i32, i64, i32, i32, f32, _vpp, _vpp,
                                           _vp, _vp, _vp, _vp, _vp]
     lib.qknorm_fwd_sharded_ex.restype = ctypes.c_int
+    lib.qknorm_fwd_e4m3.argtypes = lib.qknorm_fwd_ex.argtypes
+    lib.qknorm_fwd_e4m3.restype = ctypes.c_int
+    lib.qknorm_fwd_sharded_e4m3.argtypes = lib.qknorm_fwd_sharded_ex.argtypes
+    lib.qknorm_fwd_sharded_e4m3.restype = ctypes.c_int
     lib.qknorm_status_string.argtypes = [ctypes.c_int]
     lib.qknorm_status_string.restype = ctypes.c_char_p
     lib.qknorm_device_error_word.argtypes = [ctypes.POINTER(ctypes.c_int)]
@@ -126,14 +132,31 @@ def _array(ts: Optional[Sequence[torch.Tensor]], n: int):
     return (ctypes.c_void_p * n)(*[_ptr(t) for t in ts])
 
 
+def qknorm_fwd_e4m3(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=None, *,
+                    rstd_q=None, rstd_k=None, stream=None):
+    """qknorm_fwd_e4m3: as qknorm_fwd with q, k and the outputs torch.float8_e4m3fn (gamma bf16)."""
+    return qknorm_fwd(q, k, gamma_q, gamma_k, eps, out_q, out_k, rstd_q=rstd_q, rstd_k=rstd_k,
+                      stream=stream, _act=torch.float8_e4m3fn)
+
+
+def qknorm_fwd_sharded_e4m3(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: float,
+                            out_q_shards=None, out_k_shards=None, *, partials_q=None, partials_k=None,
+                            rstd_q=None, rstd_k=None, stream=None):
+    """qknorm_fwd_sharded_e4m3: as qknorm_fwd_sharded with float8_e4m3fn activations."""
+    return qknorm_fwd_sharded(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps, out_q_shards,
+                              out_k_shards, partials_q=partials_q, partials_k=partials_k, rstd_q=rstd_q,
+                              rstd_k=rstd_k, stream=stream, _act=torch.float8_e4m3fn)
+
+
 def qknorm_fwd(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=None, *,
-               rstd_q=None, rstd_k=None, stream=None):
+               rstd_q=None, rstd_k=None, stream=None, _act=torch.bfloat16):
     """qknorm_fwd / qknorm_fwd_ex.  q [T,dq], k [T,dk] bf16 CUDA tensors (either may
     be None to skip that tensor); out_* default to new tensors, and may be the
     inputs themselves (in place).  Passing rstd_* (fp32 [T]) selects the _ex form.
     Returns (out_q, out_k)."""
     lib = load()
     bf = torch.bfloat16
+    act = _act
     ref = q if q is not None else k
     if ref is None:
         raise QKNormError(QKNORM_ERR_NULL, "q and k are both None")
@@ -141,15 +164,15 @@ def qknorm_fwd(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=None, *,
     dq = q.shape[1] if q is not None else 0
     dk = k.shape[1] if k is not None else 0
     if q is not None:
-        _expect(q, (T, dq), bf, "q")
+        _expect(q, (T, dq), act, "q")
         _expect(gamma_q, (dq,), bf, "gamma_q")
         out_q = torch.empty_like(q) if out_q is None else out_q
-        _expect(out_q, (T, dq), bf, "out_q")
+        _expect(out_q, (T, dq), act, "out_q")
     if k is not None:
-        _expect(k, (T, dk), bf, "k")
+        _expect(k, (T, dk), act, "k")
         _expect(gamma_k, (dk,), bf, "gamma_k")
         out_k = torch.empty_like(k) if out_k is None else out_k
-        _expect(out_k, (T, dk), bf, "out_k")
+        _expect(out_k, (T, dk), act, "out_k")
     if rstd_q is not None:
         _expect(rstd_q, (T,), torch.float32, "rstd_q")
     if rstd_k is not None:
@@ -157,7 +180,9 @@ def qknorm_fwd(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=None, *,
     args = [_ptr(q), _ptr(k), _ptr(gamma_q) if q is not None else None,
             _ptr(gamma_k) if k is not None else None, T, dq, dk, float(eps),
             _ptr(out_q) if q is not None else None, _ptr(out_k) if k is not None else None]
-    if rstd_q is None and rstd_k is None:
+    if act is not bf:
+        _check(lib.qknorm_fwd_e4m3(*args, _ptr(rstd_q), _ptr(rstd_k), _stream(stream)))
+    elif rstd_q is None and rstd_k is None:
         _check(lib.qknorm_fwd(*args, _stream(stream)))
     else:
         _check(lib.qknorm_fwd_ex(*args, _ptr(rstd_q), _ptr(rstd_k), _stream(stream)))
@@ -166,13 +191,14 @@ def qknorm_fwd(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=None, *,
 
 def qknorm_fwd_sharded(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: float,
                        out_q_shards=None, out_k_shards=None, *, partials_q=None, partials_k=None,
-                       rstd_q=None, rstd_k=None, stream=None):
+                       rstd_q=None, rstd_k=None, stream=None, _act=torch.bfloat16):
     """qknorm_fwd_sharded / qknorm_fwd_sharded_ex.  *_shards are lists of S CUDA
     tensors ([T, dq/S], [T, dk/S], [dq/S], [dk/S]); q_shards or k_shards may be
     None to skip that tensor.  Passing partials_* (fp32 [S,T]) or rstd_* (fp32
     [T]) selects the _ex form.  Returns (out_q_shards, out_k_shards)."""
     lib = load()
     bf = torch.bfloat16
+    act = _act
     ref = q_shards if q_shards is not None else k_shards
     if ref is None:
         raise QKNormError(QKNORM_ERR_NULL, "q_shards and k_shards are both None")
@@ -191,9 +217,9 @@ def qknorm_fwd_sharded(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: 
         if len(xs) != S or len(gs) != S or len(outs) != S:
             raise QKNormError(QKNORM_ERR_SHARDS, f"{name}: every list must hold {S} shards")
         for s in range(S):
-            _expect(xs[s], (T, w), bf, f"{name}_shards[{s}]")
+            _expect(xs[s], (T, w), act, f"{name}_shards[{s}]")
             _expect(gs[s], (w,), bf, f"gamma_{name}_shards[{s}]")
-            _expect(outs[s], (T, w), bf, f"out_{name}_shards[{s}]")
+            _expect(outs[s], (T, w), act, f"out_{name}_shards[{s}]")
         return xs, gs, outs
 
     q_shards, gamma_q_shards, out_q_shards = side(q_shards, gamma_q_shards, out_q_shards, wq, "q")
@@ -204,7 +230,10 @@ def qknorm_fwd_sharded(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: 
             _expect(t, shp, torch.float32, nm)
     args = [_array(q_shards, S), _array(k_shards, S), _array(gamma_q_shards, S), _array(gamma_k_shards, S),
             S, T, wq * S, wk * S, float(eps), _array(out_q_shards, S), _array(out_k_shards, S)]
-    if all(t is None for t in (partials_q, partials_k, rstd_q, rstd_k)):
+    if act is not bf:
+        _check(lib.qknorm_fwd_sharded_e4m3(*args, _ptr(partials_q), _ptr(partials_k), _ptr(rstd_q),
+                                           _ptr(rstd_k), _stream(stream)))
+    elif all(t is None for t in (partials_q, partials_k, rstd_q, rstd_k)):
         _check(lib.qknorm_fwd_sharded(*args, _stream(stream)))
     else:
         _check(lib.qknorm_fwd_sharded_ex(*args, _ptr(partials_q), _ptr(partials_k), _ptr(rstd_q),

@@ -47,7 +47,9 @@ def _units() -> List[Tuple[str, str, List[str]]]:
     for n in CHUNKS_PER_THREAD:
         units.append((f"qknorm_rows_n{n}.o", os.path.join(CSRC, "qknorm_rows_inst.cu"), [f"-DQKNORM_N={n}"]))
     for l in CHUNK_SLOTS_PER_LANE:
-        units.append((f"qknorm_warp_l{l}.o", os.path.join(CSRC, "qknorm_warp_inst.cu"), [f"-DQKNORM_L={l}"]))
+        for io, tag in (("IoBf16", "bf16"), ("IoE4m3", "e4m3")):
+            units.append((f"qknorm_warp_{tag}_l{l}.o", os.path.join(CSRC, "qknorm_warp_inst.cu"),
+                          [f"-DQKNORM_L={l}", f"-DQKNORM_IO={io}", f"-DQKNORM_IO_TAG={tag}"]))
     return units
 
 

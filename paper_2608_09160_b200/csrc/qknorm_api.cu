@@ -17,19 +17,19 @@
 namespace qknorm {
 
 // per-N factories, defined in qknorm_rows_inst.cu (one translation unit per N)
-#define QKNORM_DECL_N(n)        \
-  RowsKernel rows_kernel_n##n(); \
+#define QKNORM_DECL_N(n)                       \
+  RowsKernel rows_kernel_n##n(int elem_bytes); \
   RingKernel ring_kernel_n##n();
 QKNORM_DECL_N(1) QKNORM_DECL_N(2) QKNORM_DECL_N(3) QKNORM_DECL_N(4) QKNORM_DECL_N(6) QKNORM_DECL_N(8)
 
-RowsKernel rows_kernel_for(int n) {
+RowsKernel rows_kernel_for(int n, int elem_bytes) {
   switch (n) {
-    case 1: return rows_kernel_n1();
-    case 2: return rows_kernel_n2();
-    case 3: return rows_kernel_n3();
-    case 4: return rows_kernel_n4();
-    case 6: return rows_kernel_n6();
-    case 8: return rows_kernel_n8();
+    case 1: return rows_kernel_n1(elem_bytes);
+    case 2: return rows_kernel_n2(elem_bytes);
+    case 3: return rows_kernel_n3(elem_bytes);
+    case 4: return rows_kernel_n4(elem_bytes);
+    case 6: return rows_kernel_n6(elem_bytes);
+    case 8: return rows_kernel_n8(elem_bytes);
     default: return nullptr;
   }
 }
@@ -46,8 +46,10 @@ RingKernel ring_kernel_for(int n) {
   }
 }
 
-// per-L factories, defined in qknorm_warp_inst.cu (one translation unit per L)
-#define QKNORM_DECL_L(l) WarpKernel warp_kernel_l##l(bool exact);
+// per-(L, format) factories, defined in qknorm_warp_inst.cu (one translation unit each)
+#define QKNORM_DECL_L(l)                     \
+  WarpKernel warp_kernel_bf16_l##l(bool exact); \
+  WarpKernel warp_kernel_e4m3_l##l(bool exact);
 QKNORM_DECL_L(4) QKNORM_DECL_L(8) QKNORM_DECL_L(12) QKNORM_DECL_L(16) QKNORM_DECL_L(20)
 QKNORM_DECL_L(24) QKNORM_DECL_L(28) QKNORM_DECL_L(32) QKNORM_DECL_L(36) QKNORM_DECL_L(40)
 
@@ -56,20 +58,15 @@ int warp_round_up_l(int n) {
   return ((n + 3) / 4) * 4;
 }
 
-WarpKernel warp_kernel_for(int l, bool exact) {
+WarpKernel warp_kernel_for(int l, bool exact, int elem_bytes) {
+#define QKNORM_CASE_L(l) \
+  case l: return elem_bytes == 1 ? warp_kernel_e4m3_l##l(exact) : warp_kernel_bf16_l##l(exact);
   switch (l) {
-    case 4: return warp_kernel_l4(exact);
-    case 8: return warp_kernel_l8(exact);
-    case 12: return warp_kernel_l12(exact);
-    case 16: return warp_kernel_l16(exact);
-    case 20: return warp_kernel_l20(exact);
-    case 24: return warp_kernel_l24(exact);
-    case 28: return warp_kernel_l28(exact);
-    case 32: return warp_kernel_l32(exact);
-    case 36: return warp_kernel_l36(exact);
-    case 40: return warp_kernel_l40(exact);
+    QKNORM_CASE_L(4) QKNORM_CASE_L(8) QKNORM_CASE_L(12) QKNORM_CASE_L(16) QKNORM_CASE_L(20)
+    QKNORM_CASE_L(24) QKNORM_CASE_L(28) QKNORM_CASE_L(32) QKNORM_CASE_L(36) QKNORM_CASE_L(40)
     default: return nullptr;
   }
+#undef QKNORM_CASE_L
 }
 
 // Set by a ring kernel whose bounded wait ran out (0 = never happened).
@@ -136,10 +133,10 @@ int check_alias(const Params& P, int64_t T) {
   const TensorArgs* ts[2] = {&P.q, &P.k};
   for (const TensorArgs* a : ts) {
     if (a->d == 0) continue;
-    const uintptr_t row_bytes = (uintptr_t)a->w * 2u;
+    const uintptr_t row_bytes = (uintptr_t)a->w * (uintptr_t)P.elem_bytes;
     for (int s = 0; s < P.S; ++s) {
       in[n] = {(uintptr_t)a->x[s], (uintptr_t)a->x[s] + row_bytes * (uintptr_t)T};
-      gm[n] = {(uintptr_t)a->gamma[s], (uintptr_t)a->gamma[s] + row_bytes};
+      gm[n] = {(uintptr_t)a->gamma[s], (uintptr_t)a->gamma[s] + (uintptr_t)a->w * 2u};
       out[n] = {(uintptr_t)a->y[s], (uintptr_t)a->y[s] + row_bytes * (uintptr_t)T};
       ++n;
     }
@@ -171,7 +168,7 @@ bool vector_path_ok(const Params& P) {
   const TensorArgs* ts[2] = {&P.q, &P.k};
   for (const TensorArgs* a : ts) {
     if (a->d == 0) continue;
-    if (a->w % 8 != 0) return false;
+    if ((a->w * P.elem_bytes) % 16 != 0) return false;
     for (int s = 0; s < P.S; ++s)
       if (!aligned16(a->x[s]) || !aligned16(a->gamma[s]) || !aligned16(a->y[s])) return false;
   }
@@ -200,7 +197,7 @@ inline int round_up(int v, int m) { return ((v + m - 1) / m) * m; }
 //  latency (few tokens): as few chunks per thread as possible, so that one load
 //              round trip covers the row.
 bool plan_rows(const Params& P, bool latency, RowsPlan* plan) {
-  const int cq = P.q.d ? P.q.w / 8 : 0, ck = P.k.d ? P.k.w / 8 : 0;
+  const int cq = P.q.d ? P.q.w * P.elem_bytes / 16 : 0, ck = P.k.d ? P.k.w * P.elem_bytes / 16 : 0;
   const int force_n = env_int("QKNORM_FORCE_N", 0);
   const int force_sub = env_int("QKNORM_FORCE_SUB", 0);
   const int ns[] = {1, 2, 3, 4, 6, 8};
@@ -318,6 +315,7 @@ int finish_launch(const char* variant) {
 int launch_ring(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* done) {
   *done = false;
   RowsPlan plan;
+  if (P.elem_bytes != 2) return QKNORM_OK;  // bf16 only
   if (!plan_rows(P, /*latency=*/false, &plan)) return QKNORM_OK;
   RingKernel fn = ring_kernel_for(plan.n);
   if (!fn) return QKNORM_OK;
@@ -364,7 +362,7 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   int log_g = 5;
   while ((P.S << log_g) > 32) --log_g;  // g = largest power of two <= 32 / S
   const int g = 1 << log_g;
-  const int cq = P.q.d ? P.q.w / 8 : 0, ck = P.k.d ? P.k.w / 8 : 0;
+  const int cq = P.q.d ? P.q.w * P.elem_bytes / 16 : 0, ck = P.k.d ? P.k.w * P.elem_bytes / 16 : 0;
   WarpArgs wa;
   wa.log_g = log_g;
   wa.nq = (cq + g - 1) / g;
@@ -373,12 +371,12 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   const int l = warp_round_up_l(wa.nq4 + wa.nk);
   if (l < 0) return QKNORM_OK;
   const bool exact = (P.S << log_g) == 32 && cq % g == 0 && ck % g == 0 && wa.nq % 4 == 0 && wa.nk % 4 == 0;
-  WarpKernel fn = warp_kernel_for(l, exact);
+  WarpKernel fn = warp_kernel_for(l, exact, P.elem_bytes);
   if (!fn) return QKNORM_OK;
   // stage layout: Q slices, K slices (each slice row followed by the bank skew), 16 zero bytes
   const int skew = (P.S > 1 && g < 8) ? g * 16 : 0;
-  wa.q_slice_stride = cq ? P.q.w * 2 + skew : 0;
-  wa.k_slice_stride = ck ? P.k.w * 2 + skew : 0;
+  wa.q_slice_stride = cq ? P.q.w * P.elem_bytes + skew : 0;
+  wa.k_slice_stride = ck ? P.k.w * P.elem_bytes + skew : 0;
   wa.k_base = P.S * wa.q_slice_stride;
   wa.zero_off = wa.k_base + P.S * wa.k_slice_stride;
   wa.stage_bytes = round_up(wa.zero_off + 16, 128);
@@ -392,9 +390,10 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   int warps = env_int("QKNORM_WARPS", (per_sm + ctas_per_sm - 1) / ctas_per_sm);
   if (warps < 1) warps = 1;
   if (warps > kWarpMaxCtaWarps) warps = kWarpMaxCtaWarps;
-  while (warps > 1 && warps * wa.stage_bytes + l * 512 + 1024 > dev.smem_per_block) --warps;
+  const int static_smem = l * 512 * (P.elem_bytes == 1 ? 2 : 1) + 1024;  // gamma + barriers
+  while (warps > 1 && warps * wa.stage_bytes + static_smem > dev.smem_per_block) --warps;
   const int smem = warps * wa.stage_bytes;
-  if (smem + l * 512 + 1024 > dev.smem_per_block) return QKNORM_OK;
+  if (smem + static_smem > dev.smem_per_block) return QKNORM_OK;
   int rc = allow_dynamic_smem((const void*)fn, smem);
   if (rc != QKNORM_OK) return rc;
   int bres = 1;
@@ -435,7 +434,7 @@ int launch(Params& P, cudaStream_t stream) {
     }
     RowsPlan plan;
     if (plan_rows(P, latency, &plan)) {
-      RowsKernel fn = rows_kernel_for(plan.n);
+      RowsKernel fn = rows_kernel_for(plan.n, P.elem_bytes);
       int bres = 1;
       rc = resident_blocks((const void*)fn, plan.threads, 0, &bres);
       if (rc != QKNORM_OK) return rc;
@@ -448,17 +447,18 @@ int launch(Params& P, cudaStream_t stream) {
       return finish_launch("rows");
     }
   }
+  void (*gen)(const Params) = P.elem_bytes == 1 ? general_kernel<IoE4m3> : general_kernel<IoBf16>;
   int bres = 1;
-  rc = resident_blocks((const void*)general_kernel, kGeneralThreads, 0, &bres);
+  rc = resident_blocks((const void*)gen, kGeneralThreads, 0, &bres);
   if (rc != QKNORM_OK) return rc;
   long long grid = (long long)bres * sms;
   if (grid > 2 * P.T) grid = 2 * P.T;
-  general_kernel<<<(unsigned)grid, kGeneralThreads, 0, stream>>>(P);
+  gen<<<(unsigned)grid, kGeneralThreads, 0, stream>>>(P);
   return finish_launch("general");
 }
 
 // Shared body of the four entry points.  Pointer arrays are host arrays of S entries.
-int run(const void* const* q, const void* const* k, const void* const* gq, const void* const* gk,
+int run(int elem_bytes, const void* const* q, const void* const* k, const void* const* gq, const void* const* gk,
         int32_t S, int64_t T, int32_t dq, int32_t dk, float eps, void* const* oq, void* const* ok,
         float* partials_q, float* partials_k, float* rstd_q, float* rstd_k, void* stream) {
   if (S < 1 || S > kMaxShards) return QKNORM_ERR_SHARDS;
@@ -476,6 +476,7 @@ int run(const void* const* q, const void* const* k, const void* const* gq, const
   P.S = S;
   P.eps = eps;
   P.log_sub = 5;
+  P.elem_bytes = elem_bytes;
   struct Side {
     TensorArgs* a;
     const void* const* x;
@@ -492,10 +493,11 @@ int run(const void* const* q, const void* const* k, const void* const* gq, const
     if (sd.d == 0) continue;
     for (int s = 0; s < S; ++s) {
       if (!sd.x[s] || !sd.g[s] || !sd.y[s]) return QKNORM_ERR_NULL;
-      if ((((uintptr_t)sd.x[s]) | ((uintptr_t)sd.g[s]) | ((uintptr_t)sd.y[s])) & 1u) return QKNORM_ERR_ALIGN;
-      sd.a->x[s] = (const uint16_t*)sd.x[s];
+      if (((uintptr_t)sd.g[s]) & 1u) return QKNORM_ERR_ALIGN;
+      if (elem_bytes == 2 && ((((uintptr_t)sd.x[s]) | ((uintptr_t)sd.y[s])) & 1u)) return QKNORM_ERR_ALIGN;
+      sd.a->x[s] = sd.x[s];
       sd.a->gamma[s] = (const uint16_t*)sd.g[s];
-      sd.a->y[s] = (uint16_t*)sd.y[s];
+      sd.a->y[s] = sd.y[s];
     }
     if ((((uintptr_t)sd.partials) | ((uintptr_t)sd.rstd)) & 3u) return QKNORM_ERR_ALIGN;
     sd.a->partials = sd.partials;
@@ -513,14 +515,14 @@ extern "C" {
 
 int qknorm_fwd(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
                int32_t dq, int32_t dk, float eps, void* out_q, void* out_k, void* stream) {
-  return qknorm::run(&q, &k, &gamma_q, &gamma_k, 1, tokens, dq, dk, eps, &out_q, &out_k, nullptr, nullptr,
+  return qknorm::run(2, &q, &k, &gamma_q, &gamma_k, 1, tokens, dq, dk, eps, &out_q, &out_k, nullptr, nullptr,
                      nullptr, nullptr, stream);
 }
 
 int qknorm_fwd_ex(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
                   int32_t dq, int32_t dk, float eps, void* out_q, void* out_k, float* rstd_q, float* rstd_k,
                   void* stream) {
-  return qknorm::run(&q, &k, &gamma_q, &gamma_k, 1, tokens, dq, dk, eps, &out_q, &out_k, nullptr, nullptr,
+  return qknorm::run(2, &q, &k, &gamma_q, &gamma_k, 1, tokens, dq, dk, eps, &out_q, &out_k, nullptr, nullptr,
                      rstd_q, rstd_k, stream);
 }
 
@@ -528,7 +530,7 @@ int qknorm_fwd_sharded(const void* const* q_shards, const void* const* k_shards,
                        const void* const* gamma_q_shards, const void* const* gamma_k_shards,
                        int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
                        void* const* out_q_shards, void* const* out_k_shards, void* stream) {
-  return qknorm::run(q_shards, k_shards, gamma_q_shards, gamma_k_shards, num_shards, tokens, dq, dk, eps,
+  return qknorm::run(2, q_shards, k_shards, gamma_q_shards, gamma_k_shards, num_shards, tokens, dq, dk, eps,
                      out_q_shards, out_k_shards, nullptr, nullptr, nullptr, nullptr, stream);
 }
 
@@ -537,7 +539,23 @@ int qknorm_fwd_sharded_ex(const void* const* q_shards, const void* const* k_shar
                           int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
                           void* const* out_q_shards, void* const* out_k_shards, float* partials_q,
                           float* partials_k, float* rstd_q, float* rstd_k, void* stream) {
-  return qknorm::run(q_shards, k_shards, gamma_q_shards, gamma_k_shards, num_shards, tokens, dq, dk, eps,
+  return qknorm::run(2, q_shards, k_shards, gamma_q_shards, gamma_k_shards, num_shards, tokens, dq, dk, eps,
+                     out_q_shards, out_k_shards, partials_q, partials_k, rstd_q, rstd_k, stream);
+}
+
+int qknorm_fwd_e4m3(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
+                    int32_t dq, int32_t dk, float eps, void* out_q, void* out_k, float* rstd_q, float* rstd_k,
+                    void* stream) {
+  return qknorm::run(1, &q, &k, &gamma_q, &gamma_k, 1, tokens, dq, dk, eps, &out_q, &out_k, nullptr, nullptr,
+                     rstd_q, rstd_k, stream);
+}
+
+int qknorm_fwd_sharded_e4m3(const void* const* q_shards, const void* const* k_shards,
+                            const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                            int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
+                            void* const* out_q_shards, void* const* out_k_shards, float* partials_q,
+                            float* partials_k, float* rstd_q, float* rstd_k, void* stream) {
+  return qknorm::run(1, q_shards, k_shards, gamma_q_shards, gamma_k_shards, num_shards, tokens, dq, dk, eps,
                      out_q_shards, out_k_shards, partials_q, partials_k, rstd_q, rstd_k, stream);
 }
 

@@ -25,6 +25,7 @@ __device__ __forceinline__ float block_sum_256(float v, float* red) {
   return tot;
 }
 
+template <class IO>
 __global__ void __launch_bounds__(kGeneralThreads) general_kernel(const __grid_constant__ Params P) {
   __shared__ float red[kGeneralThreads / 32];
   const long long items = 2 * P.T;
@@ -36,28 +37,26 @@ __global__ void __launch_bounds__(kGeneralThreads) general_kernel(const __grid_c
     // Phase A per slice, combined in ascending slice order
     float total = 0.f;
     for (int s = 0; s < P.S; ++s) {
-      const uint16_t* x = A.x[s] + t * w;
+      const long long row = t * w;
       float acc = 0.f;
       for (int j = threadIdx.x; j < w; j += kGeneralThreads) {
-        const float v = __uint_as_float(((uint32_t)x[j]) << 16);
+        const float v = IO::load(A.x[s], row + j);
         acc = fmaf(v, v, acc);
       }
       const float part = block_sum_256(acc, red);
       if (A.partials != nullptr && threadIdx.x == 0) A.partials[(long long)s * P.T + t] = part;
       total += part;
     }
-    const float r = rstd_from_sumsq(total, A.d, P.eps);
+    const float r = rstd_of(total, A.inv_d, P.eps);
     if (A.rstd != nullptr && threadIdx.x == 0) A.rstd[t] = r;
     // Phases B/C
     for (int s = 0; s < P.S; ++s) {
-      const uint16_t* x = A.x[s] + t * w;
+      const long long row = t * w;
       const uint16_t* gm = A.gamma[s];
-      uint16_t* y = A.y[s] + t * w;
       for (int j = threadIdx.x; j < w; j += kGeneralThreads) {
-        const float v = __uint_as_float(((uint32_t)x[j]) << 16);
+        const float v = IO::load(A.x[s], row + j);
         const float gv = __uint_as_float(((uint32_t)gm[j]) << 16);
-        const __nv_bfloat16 o = __float2bfloat16_rn((v * gv) * r);
-        y[j] = *reinterpret_cast<const uint16_t*>(&o);
+        IO::store(A.y[s], row + j, (v * gv) * r);
       }
     }
   }

@@ -12,9 +12,9 @@ constexpr int kMaxSlots = 64;    // shared-memory partial sums per CTA (one per 
 
 // One tensor (Q or K) held as S equal column slices.  S == 1 is the unsharded case.
 struct TensorArgs {
-  const uint16_t* x[kMaxShards];      // X_local of Algorithm 1, slice s: [T, w] bf16
+  const void* x[kMaxShards];          // X_local of Algorithm 1, slice s: [T, w] bf16 or FP8-E4M3
   const uint16_t* gamma[kMaxShards];  // W_local, slice s: [w] bf16
-  uint16_t* y[kMaxShards];            // Y_local, slice s: [T, w] bf16 (may equal x[s])
+  void* y[kMaxShards];                // Y_local, slice s: [T, w], same format as x (may equal x[s])
   float* partials;                    // optional [S, T]: Phase A scalar of every slice
   float* rstd;                        // optional [T]: RMS^-1 of Algorithm 1
   int d;                              // full width H_total (0 = tensor absent)
@@ -31,6 +31,7 @@ struct Params {
   int S;         // slices per tensor
   float eps;
   int log_sub;   // 4 or 5: lanes that reduce together by shuffle (16 or 32)
+  int elem_bytes;  // 2 = bf16 activations, 1 = FP8-E4M3 activations
 };
 
 }  // namespace qknorm

@@ -102,7 +102,7 @@ ring_kernel(const __grid_constant__ Params P, const int nst, const int stage_byt
   __shared__ __align__(8) unsigned long long bars[kRingMaxStages];
 
   const int tid = threadIdx.x;
-  const LaneMap m = make_lane(P, tid, N);
+  const LaneMap m = make_lane<IoBf16>(P, tid, N);
   const uint32_t smem0 = ptx::smem_u32(ring_smem);
   const uint32_t bar0 = ptx::smem_u32(bars);
   const uint32_t row_bytes = ((uint32_t)P.q.d + (uint32_t)P.k.d) * 2u;
@@ -150,7 +150,7 @@ ring_kernel(const __grid_constant__ Params P, const int nst, const int stage_byt
   }
 
   uint4 gm[N];
-  load_gamma<N>(m, gm);
+  load_gamma<IoBf16, N>(m, gm);
   // loop-invariant offsets inside a stage: the chunk, or the zeros behind the row
   uint32_t soff[N];
 #pragma unroll
@@ -168,11 +168,11 @@ ring_kernel(const __grid_constant__ Params P, const int nst, const int stage_byt
     uint4 v[N];
 #pragma unroll
     for (int j = 0; j < N; ++j) v[j] = ptx::lds128(base + soff[j]);
-    const float a = lane_group_sum(sumsq_chunks<N>(v), P.log_sub);  // Phase A
+    const float a = lane_group_sum(sumsq_chunks<IoBf16, N>(v), P.log_sub);  // Phase A
     if (m.leader) slots[par][m.slot] = a;
     __syncthreads();  // slots visible; the stage has been read by everyone
     if (tid < 32 && i + nst < n_my) issue(i + nst, st);
-    finish_token<N>(P, m, slots[par], v, gm, t);
+    finish_token<IoBf16, N>(P, m, slots[par], v, gm, t);
     if (++st == nst) { st = 0; phase ^= 1u; }
   }
 }

@@ -51,12 +51,13 @@ struct LaneMap {
   unsigned char* y;
   float* rstd;
   float* partials;
-  unsigned long long slice_row_bytes;  // w * 2
+  unsigned long long slice_row_bytes;  // w * bytes per element
   uint32_t chunk_off;  // g * 16: byte offset of this thread's first chunk inside its slice row
   uint32_t stride;     // G * 16: byte distance between a thread's consecutive chunks
   uint32_t stage_off;  // byte offset of the first chunk inside a gathered row (Q slices, then K slices)
 };
 
+template <class IO>
 __device__ __forceinline__ LaneMap make_lane(const Params& P, int tid, int n_chunks_per_thread) {
   LaneMap m;
   const bool is_k = P.k.d != 0 && tid >= P.k.first_thread;
@@ -67,7 +68,7 @@ __device__ __forceinline__ LaneMap make_lane(const Params& P, int tid, int n_chu
   m.active = A.d != 0 && s < P.S;
   m.slice = m.active ? s : 0;
   m.g = rel - s * G;
-  const int chunks = A.w >> 3;
+  const int chunks = (A.w * IO::kBytes) >> 4;  // 16-byte chunks per slice row
   int nv = m.active && m.g < chunks ? (chunks - m.g + G - 1) / G : 0;
   m.nvalid = nv < n_chunks_per_thread ? nv : n_chunks_per_thread;
   m.inv_d = A.inv_d;
@@ -81,30 +82,25 @@ __device__ __forceinline__ LaneMap make_lane(const Params& P, int tid, int n_chu
   m.y = reinterpret_cast<unsigned char*>(A.y[m.slice]);
   m.rstd = A.rstd;
   m.partials = A.partials;
-  m.slice_row_bytes = (unsigned long long)A.w * 2ull;
+  m.slice_row_bytes = (unsigned long long)A.w * IO::kBytes;
   m.chunk_off = (uint32_t)m.g * 16u;
   m.stride = (uint32_t)G * 16u;
-  m.stage_off = (is_k ? (uint32_t)P.q.d * 2u : 0u) + (uint32_t)m.slice * (uint32_t)A.w * 2u + m.chunk_off;
+  m.stage_off = (is_k ? (uint32_t)P.q.d * IO::kBytes : 0u) + (uint32_t)m.slice * (uint32_t)A.w * IO::kBytes + m.chunk_off;
   return m;
 }
 
-__device__ __forceinline__ float2 bf_unpack2(uint32_t u) { return make_float2(bf_lo(u), bf_hi(u)); }
-
-// Sum of squares of N chunks (zeros where a chunk is absent): two packed accumulators.
-template <int N>
+// Sum of squares of N chunks (zeros where a chunk is absent): independent accumulators per chunk pair.
+template <class IO, int N>
 __device__ __forceinline__ float sumsq_chunks(const uint4 (&v)[N]) {
-  float2 a0 = make_float2(0.f, 0.f), a1 = make_float2(0.f, 0.f);
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
   for (int i = 0; i < N; ++i) {
-    const float2 f0 = bf_unpack2(v[i].x), f1 = bf_unpack2(v[i].y);
-    const float2 f2 = bf_unpack2(v[i].z), f3 = bf_unpack2(v[i].w);
-    a0 = __ffma2_rn(f0, f0, a0);
-    a1 = __ffma2_rn(f1, f1, a1);
-    a0 = __ffma2_rn(f2, f2, a0);
-    a1 = __ffma2_rn(f3, f3, a1);
+    IO::sumsq_word(v[i].x, a0, a1);
+    IO::sumsq_word(v[i].y, a2, a3);
+    IO::sumsq_word(v[i].z, a0, a1);
+    IO::sumsq_word(v[i].w, a2, a3);
   }
-  const float2 a = __fadd2_rn(a0, a1);
-  return a.x + a.y;
+  return (a0 + a2) + (a1 + a3);
 }
 
 // Lane-group sum: every lane of a 16- or 32-lane group gets the group's total.
@@ -142,42 +138,13 @@ __device__ __forceinline__ float own_slice_scalar(const float* slots, const Lane
   return part;
 }
 
-__device__ __forceinline__ uint32_t scale_word2(uint32_t x, uint32_t g, float2 r2) {
-  const float2 o = __fmul2_rn(__fmul2_rn(bf_unpack2(x), bf_unpack2(g)), r2);
-  return bf_pack(o.x, o.y);
-}
-
-__device__ __forceinline__ uint4 scale_chunk2(const uint4& x, const uint4& g, float2 r2) {
-  uint4 o;
-  o.x = scale_word2(x.x, g.x, r2);
-  o.y = scale_word2(x.y, g.y, r2);
-  o.z = scale_word2(x.z, g.z, r2);
-  o.w = scale_word2(x.w, g.w, r2);
-  return o;
-}
-
-// The same with the mixed-precision multiply (no widening instructions).
-__device__ __forceinline__ uint32_t scale_word_mixed(uint32_t x, uint32_t g, float2 r2) {
-  const float2 o = __fmul2_rn(mul_bf16x2(x, g), r2);
-  return bf_pack(o.x, o.y);
-}
-
-__device__ __forceinline__ uint4 scale_chunk_mixed(const uint4& x, const uint4& g, float2 r2) {
-  uint4 o;
-  o.x = scale_word_mixed(x.x, g.x, r2);
-  o.y = scale_word_mixed(x.y, g.y, r2);
-  o.z = scale_word_mixed(x.z, g.z, r2);
-  o.w = scale_word_mixed(x.w, g.w, r2);
-  return o;
-}
-
 // Everything after the row is in registers and the slots are visible: combine,
 // RMS^-1, the optional statistics, scale and store.  `t` is the token.
-template <int N>
+template <class IO, int N>
 __device__ __forceinline__ void finish_token(const Params& P, const LaneMap& m, const float* slots,
-                                             const uint4 (&v)[N], const uint4 (&gm)[N], long long t) {
+                                             const uint4 (&v)[N], const uint4 (&gm)[N * IO::kGammaVecs], long long t) {
   const float total = combine_slices(slots, m, P.S);
-  const float r = rsqrtf(fmaf(total, m.inv_d, P.eps));
+  const float r = rstd_of(total, m.inv_d, P.eps);
   if (!m.active) return;
   if (m.rstd != nullptr && m.first) m.rstd[t] = r;
   if (m.partials != nullptr && m.g == 0) m.partials[(long long)m.slice * P.T + t] = own_slice_scalar(slots, m);
@@ -185,15 +152,22 @@ __device__ __forceinline__ void finish_token(const Params& P, const LaneMap& m, 
   unsigned char* out = m.y + (unsigned long long)t * m.slice_row_bytes + m.chunk_off;
 #pragma unroll
   for (int i = 0; i < N; ++i) {
-    if (i < m.nvalid) st_stream(reinterpret_cast<uint4*>(out + (size_t)i * m.stride), scale_chunk2(v[i], gm[i], r2));
+    if (i < m.nvalid)
+      st_stream(reinterpret_cast<uint4*>(out + (size_t)i * m.stride),
+                IO::scale_chunk(v[i], gm[i * IO::kGammaVecs], gm[i * IO::kGammaVecs + IO::kGammaVecs - 1], r2));
   }
 }
 
-template <int N>
-__device__ __forceinline__ void load_gamma(const LaneMap& m, uint4 (&gm)[N]) {
+// gamma for the thread's chunks: kGammaVecs 16-byte bf16 vectors per activation chunk.
+template <class IO, int N>
+__device__ __forceinline__ void load_gamma(const LaneMap& m, uint4 (&gm)[N * IO::kGammaVecs]) {
 #pragma unroll
-  for (int i = 0; i < N; ++i)
-    gm[i] = i < m.nvalid ? __ldg(m.gamma + m.g + i * (int)(m.stride >> 4)) : make_uint4(0u, 0u, 0u, 0u);
+  for (int i = 0; i < N; ++i) {
+    const int c = m.g + i * (int)(m.stride >> 4);  // the thread's i-th activation chunk inside its slice row
+#pragma unroll
+    for (int v = 0; v < IO::kGammaVecs; ++v)
+      gm[i * IO::kGammaVecs + v] = i < m.nvalid ? __ldg(m.gamma + c * IO::kGammaVecs + v) : make_uint4(0u, 0u, 0u, 0u);
+  }
 }
 
 }  // namespace qknorm

@@ -15,12 +15,12 @@
 
 namespace qknorm {
 
-template <int N>
+template <int N, class IO>
 __global__ void __launch_bounds__(max_threads_for(N), min_blocks_for(N)) rows_kernel(const __grid_constant__ Params P) {
   __shared__ __align__(16) float slots[2][kMaxSlots];
-  const LaneMap m = make_lane(P, threadIdx.x, N);
-  uint4 gm[N];
-  load_gamma<N>(m, gm);
+  const LaneMap m = make_lane<IO>(P, threadIdx.x, N);
+  uint4 gm[N * IO::kGammaVecs];
+  load_gamma<IO, N>(m, gm);
 
   int par = 0;
   for (long long t = blockIdx.x; t < P.T; t += gridDim.x, par ^= 1) {
@@ -30,14 +30,14 @@ __global__ void __launch_bounds__(max_threads_for(N), min_blocks_for(N)) rows_ke
     for (int i = 0; i < N; ++i)
       v[i] = i < m.nvalid ? ld_stream(reinterpret_cast<const uint4*>(row + (size_t)i * m.stride))
                           : make_uint4(0u, 0u, 0u, 0u);
-    const float a = lane_group_sum(sumsq_chunks<N>(v), P.log_sub);  // Phase A
+    const float a = lane_group_sum(sumsq_chunks<IO, N>(v), P.log_sub);  // Phase A
     if (m.leader) slots[par][m.slot] = a;
     __syncthreads();
-    finish_token<N>(P, m, slots[par], v, gm, t);
+    finish_token<IO, N>(P, m, slots[par], v, gm, t);
   }
 }
 
 using RowsKernel = void (*)(const Params);
-RowsKernel rows_kernel_for(int n);  // nullptr outside the instantiated set
+RowsKernel rows_kernel_for(int n, int elem_bytes);  // nullptr outside the instantiated set
 
 }  // namespace qknorm

@@ -64,11 +64,12 @@ struct WarpArgs {
 
 // EXACT: every lane has all nq / nk chunk slots (S*g == 32 and the slice rows are
 // whole multiples of g chunks), so the stores need no per-lane test either.
-template <int L, bool EXACT>
+template <int L, bool EXACT, class IO>
 __global__ void __launch_bounds__(kWarpMaxCtaWarps * 32, warp_min_blocks(L))
 warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs wa) {
+  constexpr int GV = IO::kGammaVecs;                            // 16-byte gamma vectors per chunk slot
   extern __shared__ __align__(128) unsigned char warp_smem[];  // one stage per warp
-  __shared__ uint4 gsm[L][32];
+  __shared__ uint4 gsm[L * GV][32];
   __shared__ __align__(8) unsigned long long bars[kWarpMaxCtaWarps];
 
   const int lane = threadIdx.x & 31;
@@ -78,7 +79,7 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   const int l = lane & (g - 1);
   const bool active = s < P.S;
   const int ss = active ? s : 0;
-  const int cq = P.q.w >> 3, ck = P.k.w >> 3;  // 16-byte chunks per slice row
+  const int cq = (P.q.w * IO::kBytes) >> 4, ck = (P.k.w * IO::kBytes) >> 4;  // 16-byte chunks per slice row
   const int nvq = EXACT ? wa.nq : ((active && l < cq) ? (cq - l + g - 1) / g : 0);
   const int nvk = EXACT ? wa.nk : ((active && l < ck) ? (ck - l + g - 1) / g : 0);
   const int n_slots = wa.nq4 + wa.nk;  // uniform
@@ -100,13 +101,13 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   if (lane < 2 * P.S) {
     const TensorArgs& A = issue_q ? P.q : P.k;
     if (A.d != 0) {
-      my_bytes = (uint32_t)A.w * 2u;
+      my_bytes = (uint32_t)A.w * IO::kBytes;
       my_src = reinterpret_cast<const unsigned char*>(A.x[is]);
       my_dst = issue_q ? (uint32_t)is * (uint32_t)wa.q_slice_stride
                        : (uint32_t)wa.k_base + (uint32_t)is * (uint32_t)wa.k_slice_stride;
     }
   }
-  const uint32_t row_bytes = ((uint32_t)P.q.d + (uint32_t)P.k.d) * 2u;
+  const uint32_t row_bytes = ((uint32_t)P.q.d + (uint32_t)P.k.d) * IO::kBytes;
   const uint64_t policy = ptx::policy_evict_first();
   auto arm = [&](long long t) {  // whole warp
     if (lane == 0) ptx::mbar_arrive_expect_tx(bar, row_bytes);
@@ -120,17 +121,20 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   __syncwarp();  // the warp's mbarrier is initialised (lane 0 did it above)
   if (first < P.T) arm(first);
 
-  // gamma, once per CTA (the first rows are already on their way): slot j of lane `lane`,
-  // the slots dealt round-robin to the CTA's warps
+  // gamma, once per CTA (the first rows are already on their way): slot j of lane `lane`
+  // holds the GV bf16 vectors that go with the lane's j-th chunk; slots dealt round-robin to the warps
   {
-    const uint4* gq = reinterpret_cast<const uint4*>(P.q.gamma[ss]) + l;
-    const uint4* gk = reinterpret_cast<const uint4*>(P.k.gamma[ss]) + l;
+    const uint4* gq = reinterpret_cast<const uint4*>(P.q.gamma[ss]) + (size_t)l * GV;
+    const uint4* gk = reinterpret_cast<const uint4*>(P.k.gamma[ss]) + (size_t)l * GV;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
     for (int j = warp; j < L; j += cta_warps) {
-      uint4 v = zero;
-      if (j < nvq) v = __ldg(gq + (size_t)j * g);
-      else if (j >= wa.nq4 && j - wa.nq4 < nvk) v = __ldg(gk + (size_t)(j - wa.nq4) * g);
-      gsm[j][lane] = v;
+#pragma unroll
+      for (int v = 0; v < GV; ++v) {
+        uint4 gv = zero;
+        if (j < nvq) gv = __ldg(gq + (size_t)j * g * GV + v);
+        else if (j >= wa.nq4 && j - wa.nq4 < nvk) gv = __ldg(gk + (size_t)(j - wa.nq4) * g * GV + v);
+        gsm[j * GV + v][lane] = gv;
+      }
     }
   }
   __syncthreads();  // the only block-level barrier
@@ -144,7 +148,7 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   const uint32_t sstride = (uint32_t)g * 16u;
   unsigned char* yq = reinterpret_cast<unsigned char*>(P.q.y[ss]) + (size_t)l * 16u;
   unsigned char* yk = reinterpret_cast<unsigned char*>(P.k.y[ss]) + (size_t)l * 16u;
-  const unsigned long long q_row = (unsigned long long)P.q.w * 2ull, k_row = (unsigned long long)P.k.w * 2ull;
+  const unsigned long long q_row = (unsigned long long)P.q.w * IO::kBytes, k_row = (unsigned long long)P.k.w * IO::kBytes;
 
   uint32_t phase = 0;
   for (long long t = first; t < P.T; t += step) {
@@ -171,22 +175,22 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
       if (jb >= n_slots) break;
       // four independent chains (one per chunk slot), two accumulators each
       float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, c4 = 0.f, c5 = 0.f, c6 = 0.f, c7 = 0.f;
-      fma_bf16x2_sq(v[jb].x, c0, c1);
-      fma_bf16x2_sq(v[jb + 1].x, c2, c3);
-      fma_bf16x2_sq(v[jb + 2].x, c4, c5);
-      fma_bf16x2_sq(v[jb + 3].x, c6, c7);
-      fma_bf16x2_sq(v[jb].y, c0, c1);
-      fma_bf16x2_sq(v[jb + 1].y, c2, c3);
-      fma_bf16x2_sq(v[jb + 2].y, c4, c5);
-      fma_bf16x2_sq(v[jb + 3].y, c6, c7);
-      fma_bf16x2_sq(v[jb].z, c0, c1);
-      fma_bf16x2_sq(v[jb + 1].z, c2, c3);
-      fma_bf16x2_sq(v[jb + 2].z, c4, c5);
-      fma_bf16x2_sq(v[jb + 3].z, c6, c7);
-      fma_bf16x2_sq(v[jb].w, c0, c1);
-      fma_bf16x2_sq(v[jb + 1].w, c2, c3);
-      fma_bf16x2_sq(v[jb + 2].w, c4, c5);
-      fma_bf16x2_sq(v[jb + 3].w, c6, c7);
+      IO::sumsq_word(v[jb].x, c0, c1);
+      IO::sumsq_word(v[jb + 1].x, c2, c3);
+      IO::sumsq_word(v[jb + 2].x, c4, c5);
+      IO::sumsq_word(v[jb + 3].x, c6, c7);
+      IO::sumsq_word(v[jb].y, c0, c1);
+      IO::sumsq_word(v[jb + 1].y, c2, c3);
+      IO::sumsq_word(v[jb + 2].y, c4, c5);
+      IO::sumsq_word(v[jb + 3].y, c6, c7);
+      IO::sumsq_word(v[jb].z, c0, c1);
+      IO::sumsq_word(v[jb + 1].z, c2, c3);
+      IO::sumsq_word(v[jb + 2].z, c4, c5);
+      IO::sumsq_word(v[jb + 3].z, c6, c7);
+      IO::sumsq_word(v[jb].w, c0, c1);
+      IO::sumsq_word(v[jb + 1].w, c2, c3);
+      IO::sumsq_word(v[jb + 2].w, c4, c5);
+      IO::sumsq_word(v[jb + 3].w, c6, c7);
       const float2 b = __fadd2_rn(__fadd2_rn(make_float2(c0, c1), make_float2(c2, c3)),
                                   __fadd2_rn(make_float2(c4, c5), make_float2(c6, c7)));
       if (jb >= wa.nq4) ak = __fadd2_rn(ak, b);
@@ -214,8 +218,8 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
     // every lane's chunks are in registers and have been used: refill the stage with the next token
     if (t + step < P.T) arm(t + step);
 
-    const float rq = rsqrtf(fmaf(totq, P.q.inv_d, P.eps));
-    const float rk = rsqrtf(fmaf(totk, P.k.inv_d, P.eps));
+    const float rq = rstd_of(totq, P.q.inv_d, P.eps);
+    const float rk = rstd_of(totk, P.k.inv_d, P.eps);
     if (lane == 0) {
       if (P.q.rstd != nullptr) P.q.rstd[t] = rq;
       if (P.k.rstd != nullptr) P.k.rstd[t] = rk;
@@ -237,7 +241,7 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
       const int nv = kpart ? (EXACT ? wa.nk : nvk) - (jb - wa.nq4) : (EXACT ? wa.nq : nvq) - jb;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint4 o = scale_chunk_mixed(v[jb + i], gsm[jb + i][lane], r2);
+        const uint4 o = IO::scale_chunk(v[jb + i], gsm[(jb + i) * GV][lane], gsm[(jb + i) * GV + GV - 1][lane], r2);
         if (i < nv) st_stream(reinterpret_cast<uint4*>(dst + (size_t)i * sstride), o);
       }
     }
@@ -245,7 +249,7 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
 }
 
 using WarpKernel = void (*)(const Params, const WarpArgs);
-WarpKernel warp_kernel_for(int l, bool exact);  // nullptr outside the instantiated set
+WarpKernel warp_kernel_for(int l, bool exact, int elem_bytes);  // nullptr outside the instantiated set
 int warp_round_up_l(int n);                      // next instantiated L >= n, or -1
 
 }  // namespace qknorm

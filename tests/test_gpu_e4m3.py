@@ -1,0 +1,128 @@
+"""GPU parity of the FP8-E4M3 entry points against the fp64 oracle (same bars as bf16:
+at most one ordinal step of the storage format from the fp64 result rounded to it,
+statistic within 1e-5)."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_09160_b200 import binding
+from paper_2608_09160_b200 import workloads as W
+from tests import gpu_harness as H
+from tests.util import e4m3_ordinal_distance
+
+pytestmark = pytest.mark.gpu
+NTHREADS = max(1, min(32, os.cpu_count() or 1))
+
+SHAPES = [
+    # name, T, dq, dk, shard counts, expected variant per shard count
+    ("e_decode", 8, 4096, 4096, (1, 4), ("rows", "rows")),
+    ("e_gqa", 900, 5120, 1024, (8, 1), ("warp", "warp")),
+    ("e_mha", 700, 5120, 5120, (4,), ("warp",)),
+    ("e_odd_width", 650, 1000, 136, (1,), ("general",)),          # not a multiple of 16 elements
+    ("e_ragged", 777, 1008, 144, (1, 3), ("warp", "warp")),       # multiples of 16, ragged over the lanes
+    ("e_tiny", 3, 16, 16, (1,), ("rows",)),
+    ("e_konly", 600, 0, 2048, (2,), ("warp",)),
+]
+
+
+def compare_e4m3(got: np.ndarray, ref: np.ndarray, what: str):
+    d = e4m3_ordinal_distance(got, ref)
+    assert int(d.max()) <= 1, f"{what}: max ordinal distance {int(d.max())}"
+    rate = float((d == 1).mean())
+    if d.size >= 4096:
+        assert rate <= 2e-3, f"{what}: {rate:.2e} of the elements are one step off"
+    return rate
+
+
+def run(w: W.Workload, S: int, in_place: bool):
+    inp = W.make_inputs_e4m3(w)
+    T = w.tokens
+    out = {}
+    stats = {}
+    names = [n for n, d in (("q", w.dq), ("k", w.dk)) if d > 0]
+    xs = {n: [t.cuda() for t in W.shard_columns(inp[n], S)] for n in names}
+    gs = {n: [t.cuda() for t in W.shard_columns(inp["gamma_" + n], S)] for n in names}
+    outs = {n: (xs[n] if in_place else [torch.full_like(t.view(torch.uint8), 0x7F).view(torch.float8_e4m3fn) for t in xs[n]])
+            for n in names}
+    rstd = {n: torch.full((T,), float("nan"), device="cuda") for n in names}
+    part = {n: torch.full((S, T), float("nan"), device="cuda") for n in names}
+    g = lambda d, n: d.get(n)
+    if S == 1:
+        binding.qknorm_fwd_e4m3(g(xs, "q")[0] if "q" in xs else None, g(xs, "k")[0] if "k" in xs else None,
+                                g(gs, "q")[0] if "q" in gs else None, g(gs, "k")[0] if "k" in gs else None, w.eps,
+                                g(outs, "q")[0] if "q" in outs else None, g(outs, "k")[0] if "k" in outs else None,
+                                rstd_q=g(rstd, "q"), rstd_k=g(rstd, "k"))
+    else:
+        binding.qknorm_fwd_sharded_e4m3(g(xs, "q"), g(xs, "k"), g(gs, "q"), g(gs, "k"), w.eps, g(outs, "q"), g(outs, "k"),
+                                        partials_q=g(part, "q"), partials_k=g(part, "k"),
+                                        rstd_q=g(rstd, "q"), rstd_k=g(rstd, "k"))
+    torch.cuda.synchronize()
+    variant = binding.last_variant()
+    for n in names:
+        xb = [W.e4m3_bits(t) for t in W.shard_columns(inp[n], S)]
+        gb = [W.bf16_bits(t) for t in W.shard_columns(inp["gamma_" + n], S)]
+        ref = oracle.rmsnorm_e4m3(xb, gb, w.eps, nthreads=NTHREADS)
+        got = np.concatenate([W.e4m3_bits(t.cpu()) for t in outs[n]], axis=1)
+        compare_e4m3(got, np.concatenate(ref["y"], axis=1), f"{w.name}/S={S}/{n}")
+        H.compare_stat(rstd[n], ref["rstd"], f"{w.name}/S={S}/rstd_{n}")
+        if S > 1:
+            H.compare_stat(part[n], ref["partials"], f"{w.name}/S={S}/partials_{n}")
+    return variant
+
+
+CASES = [(name, T, dq, dk, S, v) for name, T, dq, dk, shards, vs in SHAPES for S, v in zip(shards, vs)]
+
+
+@pytest.mark.parametrize("name,T,dq,dk,S,variant", CASES, ids=[f"{c[0]}-S{c[4]}" for c in CASES])
+@pytest.mark.parametrize("in_place", [False, True])
+def test_e4m3_matches_oracle(libqknorm, name, T, dq, dk, S, variant, in_place):
+    w = W.Workload(name, tokens=T, dq=dq, dk=dk, shards=(S,), seed=300 + len(name) + S, sigma=1.5,
+                   outlier_frac=0.01 if dq >= 4096 else 0.0)
+    assert run(w, S, in_place) == variant
+
+
+def test_e4m3_saturates_and_propagates_nan(libqknorm):
+    T, d = 4, 256
+    x = torch.zeros((T, d), dtype=torch.float32)
+    x[0, 3] = 1.0                      # one-hot: y_3 = gamma * sqrt(256) = 16 * 200 -> saturates at 448
+    x[1] = 2.0
+    x[3] = 1.0
+    x8 = x.to(torch.float8_e4m3fn)
+    bits = x8.view(torch.uint8)
+    bits[2, 7] = 0x7F                  # NaN poisons its row
+    g = torch.full((d,), 200.0, dtype=torch.bfloat16)
+    out, _ = binding.qknorm_fwd_e4m3(x8.cuda(), None, g.cuda(), None, 0.0)
+    with np.errstate(all="ignore"):
+        ref = oracle.rmsnorm_e4m3([W.e4m3_bits(x8)], [W.bf16_bits(g)], 0.0)["y"][0]
+    got = W.e4m3_bits(out.cpu())
+    assert e4m3_ordinal_distance(got, ref).max() == 0
+    assert got[0, 3] == 0x7E and (got[2] & 0x7F == 0x7F).all()
+
+
+@pytest.mark.parametrize("name", ["C3", "C4", "C5"])
+def test_full_size_e4m3(libqknorm, name):
+    w = W.WORKLOADS[name]
+    S = w.shards[-1]
+    inp = W.make_inputs_e4m3(w)
+    qs = [t.cuda() for t in W.shard_columns(inp["q"], S)]
+    ks = [t.cuda() for t in W.shard_columns(inp["k"], S)]
+    gqs = [t.cuda() for t in W.shard_columns(inp["gamma_q"], S)]
+    gks = [t.cuda() for t in W.shard_columns(inp["gamma_k"], S)]
+    oqs = qs if w.in_place else [torch.empty_like(t) for t in qs]
+    oks = ks if w.in_place else [torch.empty_like(t) for t in ks]
+    binding.qknorm_fwd_sharded_e4m3(qs, ks, gqs, gks, w.eps, oqs, oks)
+    torch.cuda.synchronize()
+    assert binding.last_variant() == "warp"
+    rng = np.random.default_rng(w.seed)
+    rows = np.unique(np.concatenate([rng.choice(w.tokens, size=2048, replace=False), [0, w.tokens - 1]]))
+    idx = torch.from_numpy(rows)
+    for nm, outs in (("q", oqs), ("k", oks)):
+        xb = [W.e4m3_bits(t[idx].contiguous()) for t in W.shard_columns(inp[nm], S)]
+        gb = [W.bf16_bits(t) for t in W.shard_columns(inp["gamma_" + nm], S)]
+        ref = oracle.rmsnorm_e4m3(xb, gb, w.eps, nthreads=NTHREADS)
+        got = np.concatenate([W.e4m3_bits(t.cpu()[idx].contiguous()) for t in outs], axis=1)
+        rate = compare_e4m3(got, np.concatenate(ref["y"], axis=1), f"{name}/e4m3/{nm}")
+        print(f"{name} e4m3 {nm}: rate at distance 1 {rate:.2e}")

@@ -383,27 +383,48 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   wa.error_word = dev.ring_error;
   // One row per warp is always in flight.  Measured on B200: throughput peaks when
   // about 76 KB of rows are in flight per SM and falls off slowly beyond that.
-  int per_sm = (76 * 1024 + wa.stage_bytes / 2) / wa.stage_bytes;
-  if (per_sm < 2) per_sm = 2;
-  if (per_sm > 16) per_sm = 16;
-  int ctas_per_sm = per_sm > kWarpMaxCtaWarps ? 2 : 1;
-  int warps = env_int("QKNORM_WARPS", (per_sm + ctas_per_sm - 1) / ctas_per_sm);
-  if (warps < 1) warps = 1;
-  if (warps > kWarpMaxCtaWarps) warps = kWarpMaxCtaWarps;
+  // FP8 rows carry twice the elements per byte and are bound by instruction issue
+  // rather than DRAM: they get half as many bytes again in flight (more warps).
+  const int in_flight = P.elem_bytes == 1 ? 114 * 1024 : 76 * 1024;
+  int rule = (in_flight + wa.stage_bytes / 2) / wa.stage_bytes;
+  if (rule < 2) rule = 2;
+  if (rule > 16) rule = 16;
+  // Among the (CTAs per SM, warps per CTA) pairs near that, prefer one whose last round of
+  // tokens is nearly full: with T / (148 * warps) rounds of several microseconds each, a
+  // half-empty last round costs short calls more than a warp more or less does.
   const int static_smem = l * 512 * (P.elem_bytes == 1 ? 2 : 1) + 1024;  // gamma + barriers
-  while (warps > 1 && warps * wa.stage_bytes + static_smem > dev.smem_per_block) --warps;
+  const int force_warps = env_int("QKNORM_WARPS", 0), force_ctas = env_int("QKNORM_CTAS_PER_SM", 0);
+  int ctas_per_sm = 0, warps = 0;
+  double best = -1.0;
+  for (int w = 1; w <= kWarpMaxCtaWarps; ++w) {
+    if (force_warps && w != force_warps) continue;
+    const int smem_w = w * wa.stage_bytes;
+    if (smem_w + static_smem > dev.smem_per_block) continue;
+    int rc = allow_dynamic_smem((const void*)fn, smem_w);
+    if (rc != QKNORM_OK) return rc;
+    int resident = 1;
+    rc = resident_blocks((const void*)fn, w * 32, smem_w, &resident);
+    if (rc != QKNORM_OK) return rc;
+    for (int c = 1; c <= resident && c <= 8; ++c) {
+      if (force_ctas && c != force_ctas && !(force_ctas > resident && c == resident)) continue;
+      const int per_sm = c * w;
+      const double rounds = (double)P.T / ((double)dev.sm_count * per_sm);
+      const double tail = rounds / (double)(long long)(rounds + 0.999999);
+      const int away = per_sm > rule ? per_sm - rule : rule - per_sm;
+      const double score = tail - 0.03 * away - 0.001 * c;
+      if (score > best) {
+        best = score;
+        ctas_per_sm = c;
+        warps = w;
+      }
+    }
+  }
+  if (warps == 0) return QKNORM_OK;  // not even one stage fits: another variant takes the call
   const int smem = warps * wa.stage_bytes;
-  if (smem + static_smem > dev.smem_per_block) return QKNORM_OK;
-  int rc = allow_dynamic_smem((const void*)fn, smem);
-  if (rc != QKNORM_OK) return rc;
-  int bres = 1;
-  rc = resident_blocks((const void*)fn, warps * 32, smem, &bres);
-  if (rc != QKNORM_OK) return rc;
-  const int cap = env_int("QKNORM_CTAS_PER_SM", ctas_per_sm);
-  if (cap > 0 && cap < bres) bres = cap;
-  long long grid = (long long)bres * dev.sm_count;  // bounded grid of co-resident CTAs
+  long long grid = (long long)ctas_per_sm * dev.sm_count;  // bounded grid of co-resident CTAs
   const long long needed = (P.T + warps - 1) / warps;
   if (grid > needed) grid = needed;
+  int rc = QKNORM_OK;
   fn<<<(unsigned)grid, warps * 32, smem, stream>>>(P, wa);
   rc = finish_launch("warp");
   *done = rc == QKNORM_OK;

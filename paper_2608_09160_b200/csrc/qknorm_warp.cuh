@@ -46,9 +46,13 @@
 
 namespace qknorm {
 
-constexpr int kWarpMaxCtaWarps = 8;  // the CTA size is a launch parameter: 1..8 warps
-// registers are shaped for this many resident CTAs of 8 warps
-__host__ __device__ constexpr int warp_min_blocks(int l) { return l <= 8 ? 4 : (l <= 16 ? 2 : 1); }
+constexpr int kWarpMaxCtaWarps = 4;  // the CTA size is a launch parameter: 1..4 warps
+// Registers are shaped for this many resident CTAs of 4 warps (64 / 128 / 168 / 255 registers
+// per thread).  FP8 rows are instruction-bound and gain from a third CTA at 17..24 slots; bf16
+// rows are faster with the registers than with the extra warps.
+__host__ __device__ constexpr int warp_min_blocks(int l, int elem_bytes) {
+  return l <= 8 ? 8 : (l <= 16 ? 4 : ((l <= 24 && elem_bytes == 1) ? 3 : 2));
+}
 
 struct WarpArgs {
   int log_g;            // log2 of the lanes per slice
@@ -65,7 +69,7 @@ struct WarpArgs {
 // EXACT: every lane has all nq / nk chunk slots (S*g == 32 and the slice rows are
 // whole multiples of g chunks), so the stores need no per-lane test either.
 template <int L, bool EXACT, class IO>
-__global__ void __launch_bounds__(kWarpMaxCtaWarps * 32, warp_min_blocks(L))
+__global__ void __launch_bounds__(kWarpMaxCtaWarps * 32, warp_min_blocks(L, IO::kBytes))
 warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs wa) {
   constexpr int GV = IO::kGammaVecs;                            // 16-byte gamma vectors per chunk slot
   extern __shared__ __align__(128) unsigned char warp_smem[];  // one stage per warp

@@ -14,4 +14,5 @@ from .qknorm_oracle import (  # noqa: F401
     e4m3_to_f64,
     f64_to_e4m3,
     rmsnorm_e4m3,
+    rmsnorm_headwise,
 )

@@ -290,6 +290,49 @@ int qko_rmsnorm_sharded_e4m3(const uint8_t* const* x_shards, const uint16_t* con
     return 0;
 }
 
+/* ---- headwise granularity (Section II-A) ------------------------------------------------------
+ *
+ * "Headwise QK-Norm computes an independent factor for each attention head": the row is cut
+ * into H/head_dim heads of head_dim consecutive elements and Eq. 1 is applied to every head on
+ * its own (mean over head_dim), with the gamma entries of those columns.  Heads never straddle
+ * a tensor-parallel shard, so the sharded form is the same computation on every shard buffer.
+ * fp8 != 0 selects FP8-E4M3 activations (x, y are bytes), else bf16 (x, y are 16-bit words).
+ * rstd (may be NULL): [T][H/head_dim]. */
+int qko_rmsnorm_headwise(const void* x, const uint16_t* gamma, int64_t T, int64_t H, int64_t head_dim,
+                         float eps, int fp8, void* y, double* y64, double* rstd, int nthreads) {
+    if (T < 0 || H < 0 || head_dim < 1 || head_dim > 4096 || (H % head_dim) != 0) return -1;
+    if (T == 0 || H == 0) return 0;
+    if (!x || !gamma) return -1;
+    const double e = (double)eps;
+    const int64_t nh = H / head_dim;
+    int nt = 1;
+#ifdef _OPENMP
+    if (nthreads > 1) nt = nthreads;
+#pragma omp parallel for num_threads(nt) schedule(static)
+#else
+    (void)nthreads;
+#endif
+    for (int64_t t = 0; t < T; ++t) {
+        for (int64_t h = 0; h < nh; ++h) {
+            const int64_t off = t * H + h * head_dim;
+            if (fp8) {
+                uint8_t head[4096];
+                const int64_t n = head_dim <= 4096 ? head_dim : 4096;   /* head_dim is validated by the caller */
+                memcpy(head, (const uint8_t*)x + off, (size_t)n);
+                rmsnorm_row_e4m3(head, gamma + h * head_dim, n, e, y ? (uint8_t*)y + off : NULL,
+                                 y64 ? y64 + off : NULL, NULL, rstd ? rstd + t * nh + h : NULL);
+            } else {
+                uint16_t head[4096];
+                const int64_t n = head_dim <= 4096 ? head_dim : 4096;
+                memcpy(head, (const uint16_t*)x + off, (size_t)n * sizeof(uint16_t));
+                rmsnorm_row(head, gamma + h * head_dim, n, e, y ? (uint16_t*)y + off : NULL,
+                            y64 ? y64 + off : NULL, NULL, rstd ? rstd + t * nh + h : NULL);
+            }
+        }
+    }
+    return 0;
+}
+
 /* Threads the OpenMP build will actually use when asked for n. */
 int qko_max_threads(void) {
 #ifdef _OPENMP

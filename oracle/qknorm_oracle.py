@@ -59,6 +59,9 @@ def _load():
         lib.qko_rmsnorm_sharded_e4m3.argtypes = [p8, pp, ctypes.c_int, ctypes.c_int64, ctypes.c_int64,
                                                  ctypes.c_float, p8, _f64p, _f64p, _f64p, _f64p, ctypes.c_int]
         lib.qko_rmsnorm_sharded_e4m3.restype = ctypes.c_int
+        lib.qko_rmsnorm_headwise.argtypes = [ctypes.c_void_p, _u16p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                             ctypes.c_float, ctypes.c_int, ctypes.c_void_p, _f64p, _f64p, ctypes.c_int]
+        lib.qko_rmsnorm_headwise.restype = ctypes.c_int
         lib.qko_max_threads.argtypes = []
         lib.qko_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -202,6 +205,33 @@ def rmsnorm_e4m3(x_shards: Sequence[np.ndarray], gamma_shards: Sequence[np.ndarr
     if rc != 0:
         raise RuntimeError(f"qko_rmsnorm_sharded_e4m3 failed ({rc})")
     res = {"y": ys, "partials": partials, "acc": acc, "rstd": rstd}
+    if want_y64:
+        res["y64"] = y64
+    return res
+
+
+def rmsnorm_headwise(x_bits: np.ndarray, gamma_bits: np.ndarray, head_dim: int, eps: float, *,
+                     want_y64: bool = False, nthreads: int = 1):
+    """Headwise granularity: Eq. 1 on every head (head_dim consecutive columns) of every row of
+    x_bits[T, H]; uint16 input = bf16, uint8 input = FP8-E4M3; gamma is bf16 [H].
+    Returns y (same dtype and shape as x_bits), rstd (fp64 [T, H/head_dim]) and, if asked, y64."""
+    lib = _load()
+    x = np.ascontiguousarray(x_bits)
+    if x.dtype not in (np.uint16, np.uint8):
+        raise TypeError("activations must be uint16 (bf16) or uint8 (E4M3) bit patterns")
+    g = _u16(gamma_bits)
+    T, H = x.shape
+    if g.shape != (H,) or head_dim < 1 or H % head_dim:
+        raise ValueError("expected gamma[H] and head_dim dividing H")
+    y = np.empty_like(x)
+    y64 = np.empty((T, H), dtype=np.float64) if want_y64 else None
+    rstd = np.empty((T, H // head_dim), dtype=np.float64)
+    rc = lib.qko_rmsnorm_headwise(x.ctypes.data, _ptr(g, _u16p), T, H, int(head_dim), float(eps),
+                                  1 if x.dtype == np.uint8 else 0, y.ctypes.data, _ptr(y64, _f64p),
+                                  _ptr(rstd, _f64p), int(nthreads))
+    if rc != 0:
+        raise RuntimeError(f"qko_rmsnorm_headwise failed ({rc})")
+    res = {"y": y, "rstd": rstd}
     if want_y64:
         res["y64"] = y64
     return res

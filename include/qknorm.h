@@ -61,7 +61,8 @@ typedef enum {
   QKNORM_ERR_ALIAS = 4,   /* an output overlaps another buffer without being exactly its own input */
   QKNORM_ERR_SHARDS = 5,  /* num_shards < 1 or > QKNORM_MAX_SHARDS */
   QKNORM_ERR_EPS = 6,     /* eps < 0 or NaN */
-  QKNORM_ERR_CUDA = 7     /* a CUDA call failed; see qknorm_last_cuda_error() */
+  QKNORM_ERR_CUDA = 7,    /* a CUDA call failed; see qknorm_last_cuda_error() */
+  QKNORM_ERR_HEADS = 8    /* head_dim < 1 or does not divide dq (or dk) */
 } qknorm_status;
 
 /*
@@ -112,6 +113,39 @@ int qknorm_fwd_sharded_ex(const void* const* q_shards, const void* const* k_shar
                           void* stream);
 
 /*
+ * qknorm_fwd_strided -- qknorm_fwd on rows that are not contiguous: row t of q starts
+ * ld_q ELEMENTS after row t-1 (ld_q >= dq), likewise k, out_q, out_k; 0 means
+ * contiguous (ld = width).  This is the layout between the projection and attention
+ * (Section II-A) when Q and K are column blocks of one fused [tokens, dq + 2*dk]
+ * projection output: q = base, k = base + dq, ld_q = ld_k = dq + 2*dk.  In place
+ * (out == in with the same ld) is allowed; the Q and K views of one buffer do not
+ * count as overlapping.  bf16; the vectorised kernels also need every ld to be a
+ * multiple of 8 elements.  A negative ld or ld < width is QKNORM_ERR_SHAPE.
+ */
+int qknorm_fwd_strided(const void* q, const void* k, const void* gamma_q, const void* gamma_k,
+                       int64_t tokens, int32_t dq, int32_t dk, int64_t ld_q, int64_t ld_k, float eps,
+                       void* out_q, void* out_k, int64_t ld_out_q, int64_t ld_out_k, void* stream);
+
+/*
+ * qknorm_fwd_headwise -- the other granularity Section II-A names: "headwise QK-Norm
+ * computes an independent factor for each attention head".  Row t of q is cut into
+ * dq/head_dim heads of head_dim consecutive columns; every head is normalised on its
+ * own, y = x / sqrt(mean over the head of x^2 + eps) * gamma, with the gamma entries of
+ * its columns (gamma_q has dq entries; tile a [head_dim] weight if the model shares
+ * it between heads).  Likewise k.  A head never straddles a tensor-parallel shard, so
+ * nothing is combined across shards: call this once per shard buffer.
+ *   ld_*            row strides in elements as in qknorm_fwd_strided (0 = contiguous)
+ *   rstd_q, rstd_k  optional [tokens, dq/head_dim] / [tokens, dk/head_dim] fp32, device
+ * bf16.  head_dim < 1 or not dividing a width is QKNORM_ERR_HEADS.  Vectorised for
+ * head_dim a multiple of 8 up to 256 with 16-byte aligned pointers and strides; any
+ * other head_dim or alignment takes a general kernel.
+ */
+int qknorm_fwd_headwise(const void* q, const void* k, const void* gamma_q, const void* gamma_k,
+                        int64_t tokens, int32_t dq, int32_t dk, int32_t head_dim,
+                        int64_t ld_q, int64_t ld_k, float eps, void* out_q, void* out_k,
+                        int64_t ld_out_q, int64_t ld_out_k, float* rstd_q, float* rstd_k, void* stream);
+
+/*
  * FP8-E4M3 activations (Section IV-C: "SwiftQK accumulates local squared sums and
  * cross-GPU scalar reductions in FP32, even for BF16 and FP8-E4M3 activations").
  * The same operation with q, k and the outputs stored as FP8 E4M3 (one byte per
@@ -147,7 +181,7 @@ int qknorm_last_cuda_error(void);
 int qknorm_device_error_word(int* out);
 
 /* Name of the kernel variant the last successful call on this thread launched
- * ("warp", "ring", "rows", "general", "none"); static storage.  For tests and benchmarks. */
+ * ("warp", "ring", "rows", "general", "head", "head_general", "none"); static storage.  For tests and benchmarks. */
 const char* qknorm_last_variant(void);
 
 /* Number of kernel launches this thread has enqueued through the library. */

@@ -22,6 +22,8 @@ EXPORTS = (
     "qknorm_fwd_ex",
     "qknorm_fwd_sharded_ex",
     "qknorm_fwd_e4m3",
+    "qknorm_fwd_strided",
+    "qknorm_fwd_headwise",
     "qknorm_fwd_sharded_e4m3",
     "qknorm_status_string",
     "qknorm_device_error_word",
@@ -39,6 +41,7 @@ QKNORM_ERR_ALIAS = 4
 QKNORM_ERR_SHARDS = 5
 QKNORM_ERR_EPS = 6
 QKNORM_ERR_CUDA = 7
+QKNORM_ERR_HEADS = 8
 
 
 class QKNormError(RuntimeError):
@@ -75,6 +78,11 @@ def load() -> ctypes.CDLL:
     lib.qknorm_fwd_e4m3.restype = ctypes.c_int
     lib.qknorm_fwd_sharded_e4m3.argtypes = lib.qknorm_fwd_sharded_ex.argtypes
     lib.qknorm_fwd_sharded_e4m3.restype = ctypes.c_int
+    lib.qknorm_fwd_strided.argtypes = [_vp, _vp, _vp, _vp, i64, i32, i32, i64, i64, f32, _vp, _vp, i64, i64, _vp]
+    lib.qknorm_fwd_strided.restype = ctypes.c_int
+    lib.qknorm_fwd_headwise.argtypes = [_vp, _vp, _vp, _vp, i64, i32, i32, i32, i64, i64, f32, _vp, _vp, i64, i64,
+                                        _vp, _vp, _vp]
+    lib.qknorm_fwd_headwise.restype = ctypes.c_int
     lib.qknorm_status_string.argtypes = [ctypes.c_int]
     lib.qknorm_status_string.restype = ctypes.c_char_p
     lib.qknorm_device_error_word.argtypes = [ctypes.POINTER(ctypes.c_int)]
@@ -239,6 +247,66 @@ def qknorm_fwd_sharded(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: 
         _check(lib.qknorm_fwd_sharded_ex(*args, _ptr(partials_q), _ptr(partials_k), _ptr(rstd_q),
                                          _ptr(rstd_k), _stream(stream)))
     return out_q_shards, out_k_shards
+
+
+def _expect_rows(t: Optional[torch.Tensor], T: int, d: int, what: str) -> int:
+    """A [T, d] bf16 CUDA view whose rows are contiguous; returns its row stride in elements."""
+    if t is None:
+        raise QKNormError(QKNORM_ERR_NULL, f"{what} is None")
+    if (not t.is_cuda or t.dtype != torch.bfloat16 or tuple(t.shape) != (T, d)
+            or (d > 1 and t.stride(1) != 1)):
+        raise QKNormError(QKNORM_ERR_SHAPE, f"{what}: expected a bf16 CUDA [{T}, {d}] view with unit column stride")
+    return int(t.stride(0)) if T > 1 else d
+
+
+def qknorm_fwd_strided(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=None, *, stream=None):
+    """qknorm_fwd_strided: q [T,dq] and k [T,dk] may be column blocks of a wider buffer
+    (row stride taken from the tensors); out_* default to the inputs (in place)."""
+    lib = load()
+    T, dq, dk = q.shape[0], q.shape[1], k.shape[1]
+    out_q = q if out_q is None else out_q
+    out_k = k if out_k is None else out_k
+    ld = [_expect_rows(q, T, dq, "q"), _expect_rows(k, T, dk, "k"),
+          _expect_rows(out_q, T, dq, "out_q"), _expect_rows(out_k, T, dk, "out_k")]
+    _expect(gamma_q, (dq,), torch.bfloat16, "gamma_q")
+    _expect(gamma_k, (dk,), torch.bfloat16, "gamma_k")
+    _check(lib.qknorm_fwd_strided(_ptr(q), _ptr(k), _ptr(gamma_q), _ptr(gamma_k), T, dq, dk, ld[0], ld[1],
+                                  float(eps), _ptr(out_q), _ptr(out_k), ld[2], ld[3], _stream(stream)))
+    return out_q, out_k
+
+
+def qknorm_fwd_headwise(q, k, gamma_q, gamma_k, head_dim: int, eps: float, out_q=None, out_k=None, *,
+                        rstd_q=None, rstd_k=None, stream=None):
+    """qknorm_fwd_headwise: every head of head_dim columns normalised on its own.  q, k are
+    [T, d] bf16 CUDA views with unit column stride (either may be None); out_* default to new
+    contiguous tensors; rstd_* are optional fp32 [T, d/head_dim]."""
+    lib = load()
+    ref = q if q is not None else k
+    if ref is None:
+        raise QKNormError(QKNORM_ERR_NULL, "q and k are both None")
+    T = ref.shape[0]
+    dq = q.shape[1] if q is not None else 0
+    dk = k.shape[1] if k is not None else 0
+    ld = [0, 0, 0, 0]
+    if q is not None:
+        out_q = torch.empty((T, dq), dtype=q.dtype, device=q.device) if out_q is None else out_q
+        ld[0], ld[2] = _expect_rows(q, T, dq, "q"), _expect_rows(out_q, T, dq, "out_q")
+        _expect(gamma_q, (dq,), torch.bfloat16, "gamma_q")
+    if k is not None:
+        out_k = torch.empty((T, dk), dtype=k.dtype, device=k.device) if out_k is None else out_k
+        ld[1], ld[3] = _expect_rows(k, T, dk, "k"), _expect_rows(out_k, T, dk, "out_k")
+        _expect(gamma_k, (dk,), torch.bfloat16, "gamma_k")
+    hd = int(head_dim)
+    if rstd_q is not None:
+        _expect(rstd_q, (T, dq // max(hd, 1)), torch.float32, "rstd_q")
+    if rstd_k is not None:
+        _expect(rstd_k, (T, dk // max(hd, 1)), torch.float32, "rstd_k")
+    _check(lib.qknorm_fwd_headwise(_ptr(q), _ptr(k), _ptr(gamma_q) if q is not None else None,
+                                   _ptr(gamma_k) if k is not None else None, T, dq, dk, hd, ld[0], ld[1],
+                                   float(eps), _ptr(out_q) if q is not None else None,
+                                   _ptr(out_k) if k is not None else None, ld[2], ld[3], _ptr(rstd_q),
+                                   _ptr(rstd_k), _stream(stream)))
+    return out_q, out_k
 
 
 def device_error_word() -> int:

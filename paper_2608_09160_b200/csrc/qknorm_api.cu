@@ -9,6 +9,7 @@
 
 #include "../../include/qknorm.h"
 #include "qknorm_general.cuh"
+#include "qknorm_head.cuh"
 #include "qknorm_params.h"
 #include "qknorm_ring.cuh"
 #include "qknorm_rows.cuh"
@@ -120,44 +121,66 @@ int current_device(const DeviceInfo** out) {
   return QKNORM_OK;
 }
 
-struct Range {
-  uintptr_t lo, hi;  // [lo, hi)
+// A buffer of the call: `rows` rows of `row_bytes` bytes, `pitch` bytes apart.
+struct Region {
+  uintptr_t base;
+  uintptr_t rows, row_bytes, pitch;
+  uintptr_t end() const { return base + (rows - 1) * pitch + row_bytes; }
 };
-inline bool overlaps(const Range& a, const Range& b) { return a.lo < b.hi && b.lo < a.hi; }
 
-// Every output range against every other range of the call.  An output may be
-// identical to its own input (same index in `in`); anything else is an error.
-int check_alias(const Params& P, int64_t T) {
-  Range in[2 * kMaxShards], gm[2 * kMaxShards], out[2 * kMaxShards], aux[4];
+// Conservative: true unless the two regions are certainly disjoint.  Strided views
+// that interleave (the Q and K columns of one fused QKV buffer) are disjoint when
+// they share the pitch and their column intervals inside a row do not meet.
+bool may_overlap(const Region& a, const Region& b) {
+  if (a.rows == 0 || b.rows == 0 || a.row_bytes == 0 || b.row_bytes == 0) return false;
+  if (a.base >= b.end() || b.base >= a.end()) return false;
+  if (a.pitch == b.pitch && a.pitch > 0 && a.row_bytes <= a.pitch && b.row_bytes <= b.pitch) {
+    const uintptr_t p = a.pitch;
+    const uintptr_t delta = b.base >= a.base ? (b.base - a.base) % p : (p - (a.base - b.base) % p) % p;
+    // inside one period a covers [0, a.row_bytes), b covers [delta, delta + b.row_bytes)
+    if (delta >= a.row_bytes && delta + b.row_bytes <= p) return false;
+  }
+  return true;
+}
+
+inline bool same_region(const Region& a, const Region& b) {
+  return a.base == b.base && a.row_bytes == b.row_bytes && (a.rows <= 1 || a.pitch == b.pitch);
+}
+
+// Every output against every other buffer of the call.  An output may be exactly
+// its own input (in place); anything else that may overlap is an error.
+int check_alias(const Params& P, int64_t T, int rstd_per_token_q = 1, int rstd_per_token_k = 1) {
+  Region in[2 * kMaxShards], gm[2 * kMaxShards], out[2 * kMaxShards], aux[4];
   int n = 0, naux = 0;
   const TensorArgs* ts[2] = {&P.q, &P.k};
+  const uintptr_t rows = (uintptr_t)T, eb = (uintptr_t)P.elem_bytes;
   for (const TensorArgs* a : ts) {
     if (a->d == 0) continue;
-    const uintptr_t row_bytes = (uintptr_t)a->w * (uintptr_t)P.elem_bytes;
+    const uintptr_t row_bytes = (uintptr_t)a->w * eb;
     for (int s = 0; s < P.S; ++s) {
-      in[n] = {(uintptr_t)a->x[s], (uintptr_t)a->x[s] + row_bytes * (uintptr_t)T};
-      gm[n] = {(uintptr_t)a->gamma[s], (uintptr_t)a->gamma[s] + (uintptr_t)a->w * 2u};
-      out[n] = {(uintptr_t)a->y[s], (uintptr_t)a->y[s] + row_bytes * (uintptr_t)T};
+      in[n] = {(uintptr_t)a->x[s], rows, row_bytes, (uintptr_t)a->ldx * eb};
+      gm[n] = {(uintptr_t)a->gamma[s], 1, (uintptr_t)a->w * 2u, (uintptr_t)a->w * 2u};
+      out[n] = {(uintptr_t)a->y[s], rows, row_bytes, (uintptr_t)a->ldy * eb};
       ++n;
     }
-    if (a->rstd) aux[naux++] = {(uintptr_t)a->rstd, (uintptr_t)a->rstd + 4u * (uintptr_t)T};
-    if (a->partials)
-      aux[naux++] = {(uintptr_t)a->partials, (uintptr_t)a->partials + 4u * (uintptr_t)T * (uintptr_t)P.S};
+    const uintptr_t rpt = (uintptr_t)(a == &P.q ? rstd_per_token_q : rstd_per_token_k);
+    if (a->rstd) aux[naux++] = {(uintptr_t)a->rstd, 1, 4u * rows * rpt, 4u * rows * rpt};
+    if (a->partials) aux[naux++] = {(uintptr_t)a->partials, 1, 4u * rows * (uintptr_t)P.S, 4u * rows * (uintptr_t)P.S};
   }
   for (int i = 0; i < n; ++i) {
     for (int j = 0; j < n; ++j) {
-      if (overlaps(out[i], gm[j])) return QKNORM_ERR_ALIAS;
-      if (overlaps(out[i], in[j]) && !(i == j && out[i].lo == in[j].lo)) return QKNORM_ERR_ALIAS;
-      if (j != i && overlaps(out[i], out[j])) return QKNORM_ERR_ALIAS;
+      if (may_overlap(out[i], gm[j])) return QKNORM_ERR_ALIAS;
+      if (may_overlap(out[i], in[j]) && !(i == j && same_region(out[i], in[j]))) return QKNORM_ERR_ALIAS;
+      if (j != i && may_overlap(out[i], out[j])) return QKNORM_ERR_ALIAS;
     }
     for (int j = 0; j < naux; ++j)
-      if (overlaps(out[i], aux[j])) return QKNORM_ERR_ALIAS;
+      if (may_overlap(out[i], aux[j])) return QKNORM_ERR_ALIAS;
   }
   for (int i = 0; i < naux; ++i) {
     for (int j = 0; j < n; ++j)
-      if (overlaps(aux[i], in[j]) || overlaps(aux[i], gm[j])) return QKNORM_ERR_ALIAS;
+      if (may_overlap(aux[i], in[j]) || may_overlap(aux[i], gm[j])) return QKNORM_ERR_ALIAS;
     for (int j = i + 1; j < naux; ++j)
-      if (overlaps(aux[i], aux[j])) return QKNORM_ERR_ALIAS;
+      if (may_overlap(aux[i], aux[j])) return QKNORM_ERR_ALIAS;
   }
   return QKNORM_OK;
 }
@@ -169,6 +192,7 @@ bool vector_path_ok(const Params& P) {
   for (const TensorArgs* a : ts) {
     if (a->d == 0) continue;
     if ((a->w * P.elem_bytes) % 16 != 0) return false;
+    if ((a->ldx * P.elem_bytes) % 16 != 0 || (a->ldy * P.elem_bytes) % 16 != 0) return false;
     for (int s = 0; s < P.S; ++s)
       if (!aligned16(a->x[s]) || !aligned16(a->gamma[s]) || !aligned16(a->y[s])) return false;
   }
@@ -481,7 +505,8 @@ int launch(Params& P, cudaStream_t stream) {
 // Shared body of the four entry points.  Pointer arrays are host arrays of S entries.
 int run(int elem_bytes, const void* const* q, const void* const* k, const void* const* gq, const void* const* gk,
         int32_t S, int64_t T, int32_t dq, int32_t dk, float eps, void* const* oq, void* const* ok,
-        float* partials_q, float* partials_k, float* rstd_q, float* rstd_k, void* stream) {
+        float* partials_q, float* partials_k, float* rstd_q, float* rstd_k, void* stream,
+        const int64_t* ld = nullptr /* {ld_q, ld_k, ld_out_q, ld_out_k}; 0 or NULL = contiguous rows */) {
   if (S < 1 || S > kMaxShards) return QKNORM_ERR_SHARDS;
   if (T < 0 || dq < 0 || dk < 0 || dq > kMaxDim || dk > kMaxDim) return QKNORM_ERR_SHAPE;
   if (dq % S != 0 || dk % S != 0) return QKNORM_ERR_SHAPE;
@@ -506,12 +531,17 @@ int run(int elem_bytes, const void* const* q, const void* const* k, const void* 
     int d;
     float* partials;
     float* rstd;
-  } sides[2] = {{&P.q, q, gq, oq, dq, partials_q, rstd_q}, {&P.k, k, gk, ok, dk, partials_k, rstd_k}};
+    int64_t ldx, ldy;
+  } sides[2] = {{&P.q, q, gq, oq, dq, partials_q, rstd_q, ld ? ld[0] : 0, ld ? ld[2] : 0},
+                {&P.k, k, gk, ok, dk, partials_k, rstd_k, ld ? ld[1] : 0, ld ? ld[3] : 0}};
   for (Side& sd : sides) {
     sd.a->d = sd.d;
     sd.a->w = sd.d / S;
     sd.a->inv_d = sd.d ? 1.0f / (float)sd.d : 0.0f;
+    sd.a->ldx = sd.ldx ? sd.ldx : sd.a->w;
+    sd.a->ldy = sd.ldy ? sd.ldy : sd.a->w;
     if (sd.d == 0) continue;
+    if (sd.a->ldx < sd.a->w || sd.a->ldy < sd.a->w) return QKNORM_ERR_SHAPE;  // rows would overlap
     for (int s = 0; s < S; ++s) {
       if (!sd.x[s] || !sd.g[s] || !sd.y[s]) return QKNORM_ERR_NULL;
       if (((uintptr_t)sd.g[s]) & 1u) return QKNORM_ERR_ALIGN;
@@ -527,6 +557,96 @@ int run(int elem_bytes, const void* const* q, const void* const* k, const void* 
   int rc = check_alias(P, T);
   if (rc != QKNORM_OK) return rc;
   return launch(P, (cudaStream_t)stream);
+}
+
+// Headwise granularity: every head of head_dim columns on its own (unsharded rows, optional strides).
+int run_headwise(const void* q, const void* k, const void* gq, const void* gk, int64_t T, int32_t dq, int32_t dk,
+                 int32_t head_dim, const int64_t* ld, float eps, void* oq, void* ok, float* rstd_q, float* rstd_k,
+                 void* stream) {
+  if (T < 0 || dq < 0 || dk < 0 || dq > kMaxDim || dk > kMaxDim) return QKNORM_ERR_SHAPE;
+  if (head_dim < 1 || dq % head_dim != 0 || dk % head_dim != 0) return QKNORM_ERR_HEADS;
+  if (!(eps >= 0.0f)) return QKNORM_ERR_EPS;
+  if (T == 0) return QKNORM_OK;
+  if (dq == 0 && dk == 0) return QKNORM_ERR_SHAPE;
+  if (dq > 0 && (!q || !gq || !oq)) return QKNORM_ERR_NULL;
+  if (dk > 0 && (!k || !gk || !ok)) return QKNORM_ERR_NULL;
+  for (int i = 0; i < 4; ++i)
+    if (ld[i] < 0) return QKNORM_ERR_SHAPE;
+  // the alias rules are those of the layerwise call on the same buffers
+  Params P;
+  memset(&P, 0, sizeof(P));
+  P.T = T;
+  P.S = 1;
+  P.elem_bytes = 2;
+  struct Side {
+    TensorArgs* a;
+    const void* x;
+    const void* g;
+    void* y;
+    int d;
+    float* rstd;
+    int64_t ldx, ldy;
+  } sides[2] = {{&P.q, q, gq, oq, dq, rstd_q, ld[0], ld[2]}, {&P.k, k, gk, ok, dk, rstd_k, ld[1], ld[3]}};
+  for (Side& sd : sides) {
+    sd.a->d = sd.a->w = sd.d;
+    sd.a->ldx = sd.ldx ? sd.ldx : sd.d;
+    sd.a->ldy = sd.ldy ? sd.ldy : sd.d;
+    if (sd.d == 0) continue;
+    if (sd.a->ldx < sd.d || sd.a->ldy < sd.d) return QKNORM_ERR_SHAPE;
+    if ((((uintptr_t)sd.x) | ((uintptr_t)sd.g) | ((uintptr_t)sd.y)) & 1u) return QKNORM_ERR_ALIGN;
+    if (((uintptr_t)sd.rstd) & 3u) return QKNORM_ERR_ALIGN;
+    sd.a->x[0] = sd.x;
+    sd.a->gamma[0] = (const uint16_t*)sd.g;
+    sd.a->y[0] = sd.y;
+    sd.a->rstd = sd.rstd;
+  }
+  int rc = check_alias(P, T, dq ? dq / head_dim : 1, dk ? dk / head_dim : 1);
+  if (rc != QKNORM_OK) return rc;
+
+  const DeviceInfo* dev = nullptr;
+  rc = current_device(&dev);
+  if (rc != QKNORM_OK) return rc;
+  HeadParams H;
+  memset(&H, 0, sizeof(H));
+  H.T = T;
+  H.head_dim = head_dim;
+  H.inv_hd = 1.0f / (float)head_dim;
+  H.eps = eps;
+  HeadSide* hs[2] = {&H.q, &H.k};
+  const TensorArgs* ts[2] = {&P.q, &P.k};
+  for (int i = 0; i < 2; ++i) {
+    hs[i]->x = ts[i]->x[0];
+    hs[i]->gamma = ts[i]->gamma[0];
+    hs[i]->y = ts[i]->y[0];
+    hs[i]->rstd = ts[i]->rstd;
+    hs[i]->ldx = ts[i]->ldx * 2;
+    hs[i]->ldy = ts[i]->ldy * 2;
+    hs[i]->nh = ts[i]->d / head_dim;
+  }
+  const char* force = getenv("QKNORM_FORCE_VARIANT");
+  const bool vec = !(force && strcmp(force, "general") == 0) && head_dim % 8 == 0 && head_dim <= 256 && vector_path_ok(P);
+  if (vec) {
+    H.hc = head_dim / 8;
+    H.log_lph = 0;
+    while ((1 << H.log_lph) < H.hc) ++H.log_lph;
+    int bres = 1;
+    rc = resident_blocks((const void*)head_kernel<4>, kHeadThreads, 0, &bres);
+    if (rc != QKNORM_OK) return rc;
+    long long grid = (long long)bres * dev->sm_count;
+    const long long needed = (T + kHeadThreads / 32 - 1) / (kHeadThreads / 32);
+    if (grid > needed) grid = needed;
+    head_kernel<4><<<(unsigned)grid, kHeadThreads, 0, (cudaStream_t)stream>>>(H);
+    return finish_launch("head");
+  }
+  int bres = 1;
+  rc = resident_blocks((const void*)head_general_kernel, kHeadThreads, 0, &bres);
+  if (rc != QKNORM_OK) return rc;
+  long long grid = (long long)bres * dev->sm_count;
+  const long long items = T * (H.q.nh + H.k.nh);
+  const long long needed = (items + kHeadThreads / 32 - 1) / (kHeadThreads / 32);
+  if (grid > needed) grid = needed;
+  head_general_kernel<<<(unsigned)grid, kHeadThreads, 0, (cudaStream_t)stream>>>(H);
+  return finish_launch("head_general");
 }
 
 }  // namespace
@@ -564,6 +684,24 @@ int qknorm_fwd_sharded_ex(const void* const* q_shards, const void* const* k_shar
                      out_q_shards, out_k_shards, partials_q, partials_k, rstd_q, rstd_k, stream);
 }
 
+int qknorm_fwd_strided(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
+                       int32_t dq, int32_t dk, int64_t ld_q, int64_t ld_k, float eps, void* out_q, void* out_k,
+                       int64_t ld_out_q, int64_t ld_out_k, void* stream) {
+  if (ld_q < 0 || ld_k < 0 || ld_out_q < 0 || ld_out_k < 0) return QKNORM_ERR_SHAPE;
+  const int64_t ld[4] = {ld_q, ld_k, ld_out_q, ld_out_k};
+  return qknorm::run(2, &q, &k, &gamma_q, &gamma_k, 1, tokens, dq, dk, eps, &out_q, &out_k, nullptr, nullptr,
+                     nullptr, nullptr, stream, ld);
+}
+
+int qknorm_fwd_headwise(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
+                        int32_t dq, int32_t dk, int32_t head_dim, int64_t ld_q, int64_t ld_k, float eps,
+                        void* out_q, void* out_k, int64_t ld_out_q, int64_t ld_out_k, float* rstd_q,
+                        float* rstd_k, void* stream) {
+  const int64_t ld[4] = {ld_q, ld_k, ld_out_q, ld_out_k};
+  return qknorm::run_headwise(q, k, gamma_q, gamma_k, tokens, dq, dk, head_dim, ld, eps, out_q, out_k, rstd_q,
+                              rstd_k, stream);
+}
+
 int qknorm_fwd_e4m3(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
                     int32_t dq, int32_t dk, float eps, void* out_q, void* out_k, float* rstd_q, float* rstd_k,
                     void* stream) {
@@ -590,6 +728,7 @@ const char* qknorm_status_string(int status) {
     case QKNORM_ERR_SHARDS: return "QKNORM_ERR_SHARDS: num_shards out of range";
     case QKNORM_ERR_EPS: return "QKNORM_ERR_EPS: eps is negative or NaN";
     case QKNORM_ERR_CUDA: return "QKNORM_ERR_CUDA: a CUDA call failed";
+    case QKNORM_ERR_HEADS: return "QKNORM_ERR_HEADS: head_dim < 1 or does not divide the width";
     default: return "unknown qknorm status";
   }
 }

@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(kGeneralThreads) general_kernel(const __grid_c
     // Phase A per slice, combined in ascending slice order
     float total = 0.f;
     for (int s = 0; s < P.S; ++s) {
-      const long long row = t * w;
+      const long long row = t * A.ldx;
       float acc = 0.f;
       for (int j = threadIdx.x; j < w; j += kGeneralThreads) {
         const float v = IO::load(A.x[s], row + j);
@@ -51,12 +51,12 @@ __global__ void __launch_bounds__(kGeneralThreads) general_kernel(const __grid_c
     if (A.rstd != nullptr && threadIdx.x == 0) A.rstd[t] = r;
     // Phases B/C
     for (int s = 0; s < P.S; ++s) {
-      const long long row = t * w;
+      const long long row = t * A.ldx, orow = t * A.ldy;
       const uint16_t* gm = A.gamma[s];
       for (int j = threadIdx.x; j < w; j += kGeneralThreads) {
         const float v = IO::load(A.x[s], row + j);
         const float gv = __uint_as_float(((uint32_t)gm[j]) << 16);
-        IO::store(A.y[s], row + j, (v * gv) * r);
+        IO::store(A.y[s], orow + j, (v * gv) * r);
       }
     }
   }

@@ -17,6 +17,8 @@ struct TensorArgs {
   void* y[kMaxShards];                // Y_local, slice s: [T, w], same format as x (may equal x[s])
   float* partials;                    // optional [S, T]: Phase A scalar of every slice
   float* rstd;                        // optional [T]: RMS^-1 of Algorithm 1
+  long long ldx;                      // elements between consecutive rows of x[s] (w when rows are contiguous)
+  long long ldy;                      // the same for y[s]
   int d;                              // full width H_total (0 = tensor absent)
   int w;                              // slice width d / S
   float inv_d;                        // 1 / H_total

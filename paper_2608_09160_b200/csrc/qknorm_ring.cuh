@@ -124,11 +124,13 @@ ring_kernel(const __grid_constant__ Params P, const int nst, const int stage_byt
   const bool issue_q = tid < P.S;
   const int is = issue_q ? tid : tid - P.S;
   uint32_t my_bytes = 0, my_dst = 0;
+  unsigned long long my_pitch = 0;  // bytes between consecutive rows of the source
   const unsigned char* my_src = nullptr;
   if (tid < 2 * P.S) {
     const TensorArgs& A = issue_q ? P.q : P.k;
     if (A.d != 0) {
       my_bytes = (uint32_t)A.w * 2u;
+      my_pitch = (unsigned long long)A.ldx * 2ull;
       my_src = reinterpret_cast<const unsigned char*>(A.x[is]);
       my_dst = (issue_q ? 0u : (uint32_t)P.q.d * 2u) + (uint32_t)is * my_bytes;
     }
@@ -140,7 +142,7 @@ ring_kernel(const __grid_constant__ Params P, const int nst, const int stage_byt
     if (tid == 0) ptx::mbar_arrive_expect_tx(bar0 + 8u * st, row_bytes);
     __syncwarp();
     if (my_bytes)
-      ptx::bulk_load(smem0 + (uint32_t)st * (uint32_t)stage_bytes + my_dst, my_src + (unsigned long long)t * my_bytes,
+      ptx::bulk_load(smem0 + (uint32_t)st * (uint32_t)stage_bytes + my_dst, my_src + (unsigned long long)t * my_pitch,
                      my_bytes, bar0 + 8u * st, policy);
   };
 

@@ -51,7 +51,8 @@ struct LaneMap {
   unsigned char* y;
   float* rstd;
   float* partials;
-  unsigned long long slice_row_bytes;  // w * bytes per element
+  unsigned long long in_pitch;   // bytes between consecutive rows of the slice's input
+  unsigned long long out_pitch;  // and of its output
   uint32_t chunk_off;  // g * 16: byte offset of this thread's first chunk inside its slice row
   uint32_t stride;     // G * 16: byte distance between a thread's consecutive chunks
   uint32_t stage_off;  // byte offset of the first chunk inside a gathered row (Q slices, then K slices)
@@ -82,7 +83,8 @@ __device__ __forceinline__ LaneMap make_lane(const Params& P, int tid, int n_chu
   m.y = reinterpret_cast<unsigned char*>(A.y[m.slice]);
   m.rstd = A.rstd;
   m.partials = A.partials;
-  m.slice_row_bytes = (unsigned long long)A.w * IO::kBytes;
+  m.in_pitch = (unsigned long long)A.ldx * IO::kBytes;
+  m.out_pitch = (unsigned long long)A.ldy * IO::kBytes;
   m.chunk_off = (uint32_t)m.g * 16u;
   m.stride = (uint32_t)G * 16u;
   m.stage_off = (is_k ? (uint32_t)P.q.d * IO::kBytes : 0u) + (uint32_t)m.slice * (uint32_t)A.w * IO::kBytes + m.chunk_off;
@@ -149,7 +151,7 @@ __device__ __forceinline__ void finish_token(const Params& P, const LaneMap& m, 
   if (m.rstd != nullptr && m.first) m.rstd[t] = r;
   if (m.partials != nullptr && m.g == 0) m.partials[(long long)m.slice * P.T + t] = own_slice_scalar(slots, m);
   const float2 r2 = make_float2(r, r);
-  unsigned char* out = m.y + (unsigned long long)t * m.slice_row_bytes + m.chunk_off;
+  unsigned char* out = m.y + (unsigned long long)t * m.out_pitch + m.chunk_off;
 #pragma unroll
   for (int i = 0; i < N; ++i) {
     if (i < m.nvalid)

@@ -25,7 +25,7 @@ __global__ void __launch_bounds__(max_threads_for(N), min_blocks_for(N)) rows_ke
   int par = 0;
   for (long long t = blockIdx.x; t < P.T; t += gridDim.x, par ^= 1) {
     uint4 v[N];
-    const unsigned char* row = m.x + (unsigned long long)t * m.slice_row_bytes + m.chunk_off;
+    const unsigned char* row = m.x + (unsigned long long)t * m.in_pitch + m.chunk_off;
 #pragma unroll
     for (int i = 0; i < N; ++i)
       v[i] = i < m.nvalid ? ld_stream(reinterpret_cast<const uint4*>(row + (size_t)i * m.stride))

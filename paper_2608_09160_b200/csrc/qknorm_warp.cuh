@@ -101,11 +101,13 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   const bool issue_q = lane < P.S;
   const int is = issue_q ? lane : lane - P.S;
   uint32_t my_bytes = 0, my_dst = 0;
+  unsigned long long my_pitch = 0;  // bytes between consecutive rows of the source
   const unsigned char* my_src = nullptr;
   if (lane < 2 * P.S) {
     const TensorArgs& A = issue_q ? P.q : P.k;
     if (A.d != 0) {
       my_bytes = (uint32_t)A.w * IO::kBytes;
+      my_pitch = (unsigned long long)A.ldx * IO::kBytes;
       my_src = reinterpret_cast<const unsigned char*>(A.x[is]);
       my_dst = issue_q ? (uint32_t)is * (uint32_t)wa.q_slice_stride
                        : (uint32_t)wa.k_base + (uint32_t)is * (uint32_t)wa.k_slice_stride;
@@ -116,7 +118,7 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   auto arm = [&](long long t) {  // whole warp
     if (lane == 0) ptx::mbar_arrive_expect_tx(bar, row_bytes);
     __syncwarp();
-    if (my_bytes) ptx::bulk_load(stage_u32 + my_dst, my_src + (unsigned long long)t * my_bytes, my_bytes, bar, policy);
+    if (my_bytes) ptx::bulk_load(stage_u32 + my_dst, my_src + (unsigned long long)t * my_pitch, my_bytes, bar, policy);
   };
 
   const int cta_warps = blockDim.x >> 5;
@@ -152,7 +154,7 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   const uint32_t sstride = (uint32_t)g * 16u;
   unsigned char* yq = reinterpret_cast<unsigned char*>(P.q.y[ss]) + (size_t)l * 16u;
   unsigned char* yk = reinterpret_cast<unsigned char*>(P.k.y[ss]) + (size_t)l * 16u;
-  const unsigned long long q_row = (unsigned long long)P.q.w * IO::kBytes, k_row = (unsigned long long)P.k.w * IO::kBytes;
+  const unsigned long long q_row = (unsigned long long)P.q.ldy * IO::kBytes, k_row = (unsigned long long)P.k.ldy * IO::kBytes;
 
   uint32_t phase = 0;
   for (long long t = first; t < P.T; t += step) {

@@ -105,3 +105,20 @@ def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "libqknorm.so"))
     with pytest.raises(binding.QKNormError, match="no fallback"):
         binding.load()
+
+
+def test_strided_and_headwise_argument_errors(libqknorm):
+    lib = libqknorm
+    strided = lambda ld_q=192, ld_k=192, oq=A, ok=A + 128, ld_oq=192, ld_ok=192, T=4: lib.qknorm_fwd_strided(
+        A, A + 128, C, D, T, 64, 32, ld_q, ld_k, 1e-6, oq, ok, ld_oq, ld_ok, None)
+    assert strided(T=0) == binding.QKNORM_OK
+    assert strided(ld_q=32) == binding.QKNORM_ERR_SHAPE                 # stride smaller than the width
+    assert strided(ld_k=-1) == binding.QKNORM_ERR_SHAPE
+    assert strided(oq=A + 64) == binding.QKNORM_ERR_ALIAS               # output columns run into the K columns
+    assert strided(oq=A, ld_oq=256) == binding.QKNORM_ERR_ALIAS         # same base, another pitch: not "in place"
+    head = lambda hd, dq=256, dk=128: lib.qknorm_fwd_headwise(A, B, C, D, 4, dq, dk, hd, 0, 0, 1e-6, E, F, 0, 0,
+                                                               None, None, None)
+    assert head(0) == binding.QKNORM_ERR_HEADS
+    assert head(96) == binding.QKNORM_ERR_HEADS                         # 256 % 96 != 0
+    assert head(64, dk=96) == binding.QKNORM_ERR_HEADS
+    assert lib.qknorm_fwd_headwise(A, B, C, D, 0, 256, 128, 64, 0, 0, 1e-6, E, F, 0, 0, None, None, None) == binding.QKNORM_OK

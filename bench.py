@@ -324,6 +324,37 @@ def config_table(steps: int, warmup: int, peak: float, skip: str):
             rows[key] = row
             del case
             torch.cuda.empty_cache()
+    rows.update(variant_rows(steps, warmup, peak))
+    return rows
+
+
+def variant_rows(steps: int, warmup: int, peak: float):
+    """The two layout/granularity variants on the C4 and C5 shapes (unsharded, bf16):
+    rows strided inside a fused [T, dq + 2*dk] projection output, and headwise (head_dim 128)."""
+    from paper_2608_09160_b200 import binding
+    rows = {}
+    for name in ("C4", "C5"):
+        w = W.WORKLOADS[name]
+        inp = W.make_inputs(w)
+        gq, gk = inp["gamma_q"].cuda(), inp["gamma_k"].cuda()
+        buf = torch.empty((w.tokens, w.dq + 2 * w.dk), dtype=torch.bfloat16, device="cuda")
+        buf[:, :w.dq] = inp["q"].cuda()
+        buf[:, w.dq:w.dq + w.dk] = inp["k"].cuda()
+        del inp
+        q, k = buf[:, :w.dq], buf[:, w.dq:w.dq + w.dk]
+        calls = {
+            f"{name}/fusedQKV-strided/in-place": lambda: binding.qknorm_fwd_strided(q, k, gq, gk, w.eps),
+            f"{name}/headwise128/fusedQKV/in-place": lambda: binding.qknorm_fwd_headwise(q, k, gq, gk, 128, w.eps, q, k),
+        }
+        for key, fn in calls.items():
+            ts = time_calls(fn, max(steps, 10), max(warmup, 3))
+            med = statistics.median(ts)
+            gbs = w.algorithmic_bytes / (med * 1e-3) / 1e9
+            rows[key] = {"us_median": round(med * 1e3, 3), "us_min": round(min(ts) * 1e3, 3), "GBps": round(gbs, 1),
+                         "frac_measured_peak": round(gbs / peak, 4), "frac_nominal_8TBps": round(gbs / NOMINAL_HBM_GBS, 4),
+                         "bytes": w.algorithmic_bytes, "variant": binding.last_variant(), "l2": "inputs larger than L2"}
+        del buf, q, k
+        torch.cuda.empty_cache()
     return rows
 
 

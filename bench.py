@@ -325,6 +325,44 @@ def config_table(steps: int, warmup: int, peak: float, skip: str):
             del case
             torch.cuda.empty_cache()
     rows.update(variant_rows(steps, warmup, peak))
+    rows.update(baseline_rows(steps, warmup, peak))
+    return rows
+
+
+def baseline_rows(steps: int, warmup: int, peak: float):
+    """The one-GPU stand-ins for the paper's comparison paths on the sharded prefill workloads,
+    next to the fused call on the same buffers: time and time relative to fused (the
+    paper's Fig. 3a normalises latency the same way).  GB/s counts the ALGORITHMIC bytes
+    of the fused op, so the stand-ins' extra traffic shows up as a lower figure."""
+    from paper_2608_09160_b200 import binding
+    rows = {}
+    for name in ("C4", "C5"):
+        w = W.WORKLOADS[name]
+        S = w.shards[-1]
+        case = DeviceCase(w, S)
+        d = case.dev
+        scratch_g = torch.empty((w.tokens * (w.dq + w.dk),), dtype=torch.bfloat16, device="cuda")
+        scratch_s = torch.empty((2 * S * w.tokens,), dtype=torch.float32, device="cuda")
+        calls = {
+            "fused": case.call,
+            "baseline-gather-then-norm": lambda: binding.qknorm_baseline_gather_then_norm(
+                d["q"], d["k"], d["gq"], d["gk"], w.eps, case.out_q, case.out_k, scratch=scratch_g),
+            "baseline-two-pass": lambda: binding.qknorm_baseline_two_pass(
+                d["q"], d["k"], d["gq"], d["gk"], w.eps, case.out_q, case.out_k, scratch=scratch_s),
+        }
+        med = {}
+        for key, fn in calls.items():
+            ts = time_calls(fn, max(steps, 10), max(warmup, 3))
+            med[key] = statistics.median(ts)
+        for key in ("baseline-gather-then-norm", "baseline-two-pass"):
+            gbs = case.bytes / (med[key] * 1e-3) / 1e9
+            rows[f"{name}/S{S}/{key}"] = {
+                "us_median": round(med[key] * 1e3, 3), "GBps": round(gbs, 1), "frac_measured_peak": round(gbs / peak, 4),
+                "fused_us_same_buffers": round(med["fused"] * 1e3, 3),
+                "time_relative_to_fused": round(med[key] / med["fused"], 3),
+                "launches_per_call": 2, "bytes": case.bytes, "variant": "baseline"}
+        del case, scratch_g, scratch_s, d
+        torch.cuda.empty_cache()
     return rows
 
 

@@ -44,6 +44,7 @@
 #ifndef QKNORM_H_
 #define QKNORM_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -62,7 +63,8 @@ typedef enum {
   QKNORM_ERR_SHARDS = 5,  /* num_shards < 1 or > QKNORM_MAX_SHARDS */
   QKNORM_ERR_EPS = 6,     /* eps < 0 or NaN */
   QKNORM_ERR_CUDA = 7,    /* a CUDA call failed; see qknorm_last_cuda_error() */
-  QKNORM_ERR_HEADS = 8    /* head_dim < 1 or does not divide dq (or dk) */
+  QKNORM_ERR_HEADS = 8,   /* head_dim < 1 or does not divide dq (or dk) */
+  QKNORM_ERR_SCRATCH = 9  /* scratch buffer NULL, too small, misaligned, or overlapping a buffer of the call */
 } qknorm_status;
 
 /*
@@ -167,6 +169,38 @@ int qknorm_fwd_sharded_e4m3(const void* const* q_shards, const void* const* k_sh
                             float* partials_q, float* partials_k, float* rstd_q, float* rstd_k,
                             void* stream);
 
+/*
+ * One-GPU stand-ins for the two conventional ways of doing tensor-parallel QK-Norm
+ * that the paper measures against (Section II-C, Section IV-A "Baselines"), for
+ * quoting the fused path in the paper's terms.  Same arguments and the same result
+ * as qknorm_fwd_sharded (bf16, contiguous rows, in place allowed), plus a scratch
+ * buffer in DEVICE memory that the caller owns; it must not overlap any buffer of
+ * the call (QKNORM_ERR_SCRATCH otherwise, also when it is NULL, misaligned or too
+ * small).  Its contents after the call are unspecified.
+ *
+ * qknorm_baseline_gather_then_norm -- "All-Gather, then RMSNorm": one kernel copies
+ *   the num_shards slices of every row side by side into scratch (full rows, what
+ *   every rank would hold after the All-Gather), then the normalisation runs with
+ *   the scratch as its input.  Two launches; every activation crosses HBM four
+ *   times.  scratch: tokens * (dq + dk) * 2 bytes, 16-byte aligned.
+ * qknorm_baseline_two_pass -- scalar aggregation without fusion: a statistics
+ *   kernel writes every slice's sum of squares to scratch (the scalars a rank would
+ *   send), a second kernel adds them in ascending slice order and scales.  Two
+ *   launches; every activation is read twice and written once.
+ *   scratch: 2 * num_shards * tokens floats.
+ */
+int qknorm_baseline_gather_then_norm(const void* const* q_shards, const void* const* k_shards,
+                                     const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                                     int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
+                                     void* const* out_q_shards, void* const* out_k_shards,
+                                     void* scratch, size_t scratch_bytes, void* stream);
+
+int qknorm_baseline_two_pass(const void* const* q_shards, const void* const* k_shards,
+                             const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                             int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
+                             void* const* out_q_shards, void* const* out_k_shards,
+                             float* scratch, size_t scratch_bytes, void* stream);
+
 /* Human-readable name of a qknorm_status (static storage, never NULL). */
 const char* qknorm_status_string(int status);
 
@@ -181,7 +215,7 @@ int qknorm_last_cuda_error(void);
 int qknorm_device_error_word(int* out);
 
 /* Name of the kernel variant the last successful call on this thread launched
- * ("warp", "ring", "rows", "general", "head", "head_general", "none"); static storage.  For tests and benchmarks. */
+ * ("warp", "ring", "rows", "general", "head", "head_general", "two_pass", "none"); static storage.  For tests and benchmarks. */
 const char* qknorm_last_variant(void);
 
 /* Number of kernel launches this thread has enqueued through the library. */

@@ -24,6 +24,8 @@ EXPORTS = (
     "qknorm_fwd_e4m3",
     "qknorm_fwd_strided",
     "qknorm_fwd_headwise",
+    "qknorm_baseline_gather_then_norm",
+    "qknorm_baseline_two_pass",
     "qknorm_fwd_sharded_e4m3",
     "qknorm_status_string",
     "qknorm_device_error_word",
@@ -42,6 +44,7 @@ QKNORM_ERR_SHARDS = 5
 QKNORM_ERR_EPS = 6
 QKNORM_ERR_CUDA = 7
 QKNORM_ERR_HEADS = 8
+QKNORM_ERR_SCRATCH = 9
 
 
 class QKNormError(RuntimeError):
@@ -83,6 +86,9 @@ def load() -> ctypes.CDLL:
     lib.qknorm_fwd_headwise.argtypes = [_vp, _vp, _vp, _vp, i64, i32, i32, i32, i64, i64, f32, _vp, _vp, i64, i64,
                                         _vp, _vp, _vp]
     lib.qknorm_fwd_headwise.restype = ctypes.c_int
+    for fn in (lib.qknorm_baseline_gather_then_norm, lib.qknorm_baseline_two_pass):
+        fn.argtypes = [_vpp, _vpp, _vpp, _vpp, i32, i64, i32, i32, f32, _vpp, _vpp, _vp, ctypes.c_size_t, _vp]
+        fn.restype = ctypes.c_int
     lib.qknorm_status_string.argtypes = [ctypes.c_int]
     lib.qknorm_status_string.restype = ctypes.c_char_p
     lib.qknorm_device_error_word.argtypes = [ctypes.POINTER(ctypes.c_int)]
@@ -307,6 +313,44 @@ def qknorm_fwd_headwise(q, k, gamma_q, gamma_k, head_dim: int, eps: float, out_q
                                    _ptr(out_k) if k is not None else None, ld[2], ld[3], _ptr(rstd_q),
                                    _ptr(rstd_k), _stream(stream)))
     return out_q, out_k
+
+
+def _baseline(entry, q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps, out_q_shards, out_k_shards,
+              scratch, stream):
+    S = len(q_shards)
+    T = q_shards[0].shape[0]
+    wq, wk = q_shards[0].shape[1], k_shards[0].shape[1]
+    bf = torch.bfloat16
+    out_q_shards = [torch.empty_like(t) for t in q_shards] if out_q_shards is None else out_q_shards
+    out_k_shards = [torch.empty_like(t) for t in k_shards] if out_k_shards is None else out_k_shards
+    for s in range(S):
+        _expect(q_shards[s], (T, wq), bf, f"q_shards[{s}]")
+        _expect(k_shards[s], (T, wk), bf, f"k_shards[{s}]")
+        _expect(gamma_q_shards[s], (wq,), bf, f"gamma_q_shards[{s}]")
+        _expect(gamma_k_shards[s], (wk,), bf, f"gamma_k_shards[{s}]")
+        _expect(out_q_shards[s], (T, wq), bf, f"out_q_shards[{s}]")
+        _expect(out_k_shards[s], (T, wk), bf, f"out_k_shards[{s}]")
+    if scratch is not None and (not scratch.is_cuda or not scratch.is_contiguous()):
+        raise QKNormError(QKNORM_ERR_SCRATCH, "scratch must be a contiguous CUDA tensor")
+    nbytes = scratch.numel() * scratch.element_size() if scratch is not None else 0
+    _check(entry(_array(q_shards, S), _array(k_shards, S), _array(gamma_q_shards, S), _array(gamma_k_shards, S),
+                 S, T, wq * S, wk * S, float(eps), _array(out_q_shards, S), _array(out_k_shards, S),
+                 _ptr(scratch), nbytes, _stream(stream)))
+    return out_q_shards, out_k_shards
+
+
+def qknorm_baseline_gather_then_norm(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: float,
+                                     out_q_shards=None, out_k_shards=None, *, scratch, stream=None):
+    """qknorm_baseline_gather_then_norm; scratch: CUDA tensor of >= T*(dq+dk)*2 bytes."""
+    return _baseline(load().qknorm_baseline_gather_then_norm, q_shards, k_shards, gamma_q_shards, gamma_k_shards,
+                     eps, out_q_shards, out_k_shards, scratch, stream)
+
+
+def qknorm_baseline_two_pass(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: float,
+                             out_q_shards=None, out_k_shards=None, *, scratch, stream=None):
+    """qknorm_baseline_two_pass; scratch: CUDA fp32 tensor of >= 2*S*T elements."""
+    return _baseline(load().qknorm_baseline_two_pass, q_shards, k_shards, gamma_q_shards, gamma_k_shards,
+                     eps, out_q_shards, out_k_shards, scratch, stream)
 
 
 def device_error_word() -> int:

@@ -8,6 +8,7 @@
 #include <mutex>
 
 #include "../../include/qknorm.h"
+#include "qknorm_baselines.cuh"
 #include "qknorm_general.cuh"
 #include "qknorm_head.cuh"
 #include "qknorm_params.h"
@@ -502,11 +503,13 @@ int launch(Params& P, cudaStream_t stream) {
   return finish_launch("general");
 }
 
-// Shared body of the four entry points.  Pointer arrays are host arrays of S entries.
-int run(int elem_bytes, const void* const* q, const void* const* k, const void* const* gq, const void* const* gk,
+// Validation shared by the entry points: fills P; *empty = true when there is nothing to do.
+// Pointer arrays are host arrays of S entries.
+int prepare(Params& P, bool* empty, int elem_bytes, const void* const* q, const void* const* k, const void* const* gq, const void* const* gk,
         int32_t S, int64_t T, int32_t dq, int32_t dk, float eps, void* const* oq, void* const* ok,
-        float* partials_q, float* partials_k, float* rstd_q, float* rstd_k, void* stream,
+        float* partials_q, float* partials_k, float* rstd_q, float* rstd_k,
         const int64_t* ld = nullptr /* {ld_q, ld_k, ld_out_q, ld_out_k}; 0 or NULL = contiguous rows */) {
+  *empty = true;
   if (S < 1 || S > kMaxShards) return QKNORM_ERR_SHARDS;
   if (T < 0 || dq < 0 || dk < 0 || dq > kMaxDim || dk > kMaxDim) return QKNORM_ERR_SHAPE;
   if (dq % S != 0 || dk % S != 0) return QKNORM_ERR_SHAPE;
@@ -516,7 +519,6 @@ int run(int elem_bytes, const void* const* q, const void* const* k, const void* 
   if (dq > 0 && (!q || !gq || !oq)) return QKNORM_ERR_NULL;
   if (dk > 0 && (!k || !gk || !ok)) return QKNORM_ERR_NULL;
 
-  Params P;
   memset(&P, 0, sizeof(P));
   P.T = T;
   P.S = S;
@@ -556,7 +558,100 @@ int run(int elem_bytes, const void* const* q, const void* const* k, const void* 
   }
   int rc = check_alias(P, T);
   if (rc != QKNORM_OK) return rc;
+  *empty = false;
+  return QKNORM_OK;
+}
+
+// The fused path: validate, then one launch.
+int run(int elem_bytes, const void* const* q, const void* const* k, const void* const* gq, const void* const* gk,
+        int32_t S, int64_t T, int32_t dq, int32_t dk, float eps, void* const* oq, void* const* ok,
+        float* partials_q, float* partials_k, float* rstd_q, float* rstd_k, void* stream,
+        const int64_t* ld = nullptr) {
+  Params P;
+  bool empty = true;
+  const int rc = prepare(P, &empty, elem_bytes, q, k, gq, gk, S, T, dq, dk, eps, oq, ok, partials_q, partials_k,
+                         rstd_q, rstd_k, ld);
+  if (rc != QKNORM_OK || empty) return rc;
   return launch(P, (cudaStream_t)stream);
+}
+
+// A scratch buffer must be non-NULL, aligned, large enough and away from every buffer of the call.
+int check_scratch(const Params& P, const void* scratch, size_t have, size_t need, size_t align) {
+  if (!scratch || have < need || (((uintptr_t)scratch) & (align - 1)) != 0) return QKNORM_ERR_SCRATCH;
+  const Region sc = {(uintptr_t)scratch, 1, (uintptr_t)need, (uintptr_t)need};
+  const TensorArgs* ts[2] = {&P.q, &P.k};
+  const uintptr_t rows = (uintptr_t)P.T, eb = (uintptr_t)P.elem_bytes;
+  for (const TensorArgs* a : ts) {
+    if (a->d == 0) continue;
+    for (int s = 0; s < P.S; ++s) {
+      const Region in = {(uintptr_t)a->x[s], rows, (uintptr_t)a->w * eb, (uintptr_t)a->ldx * eb};
+      const Region out = {(uintptr_t)a->y[s], rows, (uintptr_t)a->w * eb, (uintptr_t)a->ldy * eb};
+      const Region gm = {(uintptr_t)a->gamma[s], 1, (uintptr_t)a->w * 2u, (uintptr_t)a->w * 2u};
+      if (may_overlap(sc, in) || may_overlap(sc, out) || may_overlap(sc, gm)) return QKNORM_ERR_SCRATCH;
+    }
+    if (a->rstd && may_overlap(sc, Region{(uintptr_t)a->rstd, 1, 4u * rows, 4u * rows})) return QKNORM_ERR_SCRATCH;
+    if (a->partials) {
+      const uintptr_t n = 4u * rows * (uintptr_t)P.S;
+      if (may_overlap(sc, Region{(uintptr_t)a->partials, 1, n, n})) return QKNORM_ERR_SCRATCH;
+    }
+  }
+  return QKNORM_OK;
+}
+
+template <class K, class... Args>
+int launch_simple(K kernel, int threads, long long work_items, const DeviceInfo& dev, cudaStream_t stream,
+                  const char* variant, Args... args) {
+  int bres = 1;
+  int rc = resident_blocks((const void*)kernel, threads, 0, &bres);
+  if (rc != QKNORM_OK) return rc;
+  long long grid = (long long)bres * dev.sm_count;
+  if (grid > work_items) grid = work_items;
+  if (grid < 1) grid = 1;
+  kernel<<<(unsigned)grid, threads, 0, stream>>>(args...);
+  return finish_launch(variant);
+}
+
+// Baseline stand-in 1: copy the slices side by side into `scratch` (full rows), then normalise from there.
+int run_gather_then_norm(Params& P, void* scratch, size_t scratch_bytes, cudaStream_t stream) {
+  const size_t need = (size_t)P.T * ((size_t)P.q.d + (size_t)P.k.d) * (size_t)P.elem_bytes;
+  int rc = check_scratch(P, scratch, scratch_bytes, need, 16);
+  if (rc != QKNORM_OK) return rc;
+  const DeviceInfo* dev = nullptr;
+  rc = current_device(&dev);
+  if (rc != QKNORM_OK) return rc;
+  const bool vec = vector_path_ok(P);
+  const long long units = (long long)(need / (vec ? 16 : 1));
+  const long long ctas = (units + kBaselineThreads - 1) / kBaselineThreads;
+  rc = vec ? launch_simple(gather_kernel<true>, kBaselineThreads, ctas, *dev, stream, "gather", P, (unsigned char*)scratch)
+           : launch_simple(gather_kernel<false>, kBaselineThreads, ctas, *dev, stream, "gather", P, (unsigned char*)scratch);
+  if (rc != QKNORM_OK) return rc;
+  // the normalisation reads the gathered rows: slice s of a tensor is a column block of the scratch
+  Params G = P;
+  const long long pitch = (long long)P.q.d + P.k.d;  // elements
+  unsigned char* base = (unsigned char*)scratch;
+  for (int s = 0; s < P.S; ++s) {
+    if (P.q.d) G.q.x[s] = base + (size_t)s * P.q.w * P.elem_bytes;
+    if (P.k.d) G.k.x[s] = base + ((size_t)P.q.d + (size_t)s * P.k.w) * P.elem_bytes;
+  }
+  G.q.ldx = G.k.ldx = pitch;
+  return launch(G, stream);
+}
+
+// Baseline stand-in 2: a statistics pass that writes every slice's scalar to `scratch`, then a scale pass.
+int run_two_pass(Params& P, float* scratch, cudaStream_t stream) {
+  const DeviceInfo* dev = nullptr;
+  int rc = current_device(&dev);
+  if (rc != QKNORM_OK) return rc;
+  const bool vec = vector_path_ok(P);
+  const long long items = P.T * 2 * P.S;
+  const long long ctas = (items + kBaselineThreads / 32 - 1) / (kBaselineThreads / 32);
+  rc = vec ? launch_simple(stat_kernel<IoBf16, true>, kBaselineThreads, ctas, *dev, stream, "two_pass", P, scratch)
+           : launch_simple(stat_kernel<IoBf16, false>, kBaselineThreads, ctas, *dev, stream, "two_pass", P, scratch);
+  if (rc != QKNORM_OK) return rc;
+  return vec ? launch_simple(scale_kernel<IoBf16, true>, kBaselineThreads, ctas, *dev, stream, "two_pass", P,
+                             (const float*)scratch)
+             : launch_simple(scale_kernel<IoBf16, false>, kBaselineThreads, ctas, *dev, stream, "two_pass", P,
+                             (const float*)scratch);
 }
 
 // Headwise granularity: every head of head_dim columns on its own (unsharded rows, optional strides).
@@ -684,6 +779,35 @@ int qknorm_fwd_sharded_ex(const void* const* q_shards, const void* const* k_shar
                      out_q_shards, out_k_shards, partials_q, partials_k, rstd_q, rstd_k, stream);
 }
 
+int qknorm_baseline_gather_then_norm(const void* const* q_shards, const void* const* k_shards,
+                                     const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                                     int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
+                                     void* const* out_q_shards, void* const* out_k_shards, void* scratch,
+                                     size_t scratch_bytes, void* stream) {
+  qknorm::Params P;
+  bool empty = true;
+  const int rc = qknorm::prepare(P, &empty, 2, q_shards, k_shards, gamma_q_shards, gamma_k_shards, num_shards, tokens,
+                                 dq, dk, eps, out_q_shards, out_k_shards, nullptr, nullptr, nullptr, nullptr);
+  if (rc != QKNORM_OK || empty) return rc;
+  return qknorm::run_gather_then_norm(P, scratch, scratch_bytes, (cudaStream_t)stream);
+}
+
+int qknorm_baseline_two_pass(const void* const* q_shards, const void* const* k_shards,
+                             const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                             int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
+                             void* const* out_q_shards, void* const* out_k_shards, float* scratch,
+                             size_t scratch_bytes, void* stream) {
+  qknorm::Params P;
+  bool empty = true;
+  int rc = qknorm::prepare(P, &empty, 2, q_shards, k_shards, gamma_q_shards, gamma_k_shards, num_shards, tokens, dq,
+                           dk, eps, out_q_shards, out_k_shards, nullptr, nullptr, nullptr, nullptr);
+  if (rc != QKNORM_OK || empty) return rc;
+  const size_t need = (size_t)2 * (size_t)num_shards * (size_t)tokens * sizeof(float);
+  rc = qknorm::check_scratch(P, scratch, scratch_bytes, need, 4);
+  if (rc != QKNORM_OK) return rc;
+  return qknorm::run_two_pass(P, scratch, (cudaStream_t)stream);
+}
+
 int qknorm_fwd_strided(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
                        int32_t dq, int32_t dk, int64_t ld_q, int64_t ld_k, float eps, void* out_q, void* out_k,
                        int64_t ld_out_q, int64_t ld_out_k, void* stream) {
@@ -729,6 +853,7 @@ const char* qknorm_status_string(int status) {
     case QKNORM_ERR_EPS: return "QKNORM_ERR_EPS: eps is negative or NaN";
     case QKNORM_ERR_CUDA: return "QKNORM_ERR_CUDA: a CUDA call failed";
     case QKNORM_ERR_HEADS: return "QKNORM_ERR_HEADS: head_dim < 1 or does not divide the width";
+    case QKNORM_ERR_SCRATCH: return "QKNORM_ERR_SCRATCH: scratch buffer missing, too small, misaligned or overlapping";
     default: return "unknown qknorm status";
   }
 }

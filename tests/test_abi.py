@@ -122,3 +122,23 @@ def test_strided_and_headwise_argument_errors(libqknorm):
     assert head(96) == binding.QKNORM_ERR_HEADS                         # 256 % 96 != 0
     assert head(64, dk=96) == binding.QKNORM_ERR_HEADS
     assert lib.qknorm_fwd_headwise(A, B, C, D, 0, 256, 128, 64, 0, 0, 1e-6, E, F, 0, 0, None, None, None) == binding.QKNORM_OK
+
+
+def test_baseline_scratch_errors(libqknorm):
+    lib = libqknorm
+    arr = ctypes.c_void_p * 2
+    mk = lambda base: arr(base, base + 0x10000)
+    SC = 0x70000000
+    def two_pass(scratch, nbytes, T=4):
+        return lib.qknorm_baseline_two_pass(mk(A), mk(B), mk(C), mk(D), 2, T, 64, 64, 1e-6, mk(E), mk(F), scratch, nbytes, None)
+    def gather(scratch, nbytes, T=4):
+        return lib.qknorm_baseline_gather_then_norm(mk(A), mk(B), mk(C), mk(D), 2, T, 64, 64, 1e-6, mk(E), mk(F),
+                                                    scratch, nbytes, None)
+    assert two_pass(None, 0, T=0) == binding.QKNORM_OK
+    assert two_pass(None, 1 << 20) == binding.QKNORM_ERR_SCRATCH
+    assert two_pass(SC, 2 * 2 * 4 * 4 - 1) == binding.QKNORM_ERR_SCRATCH       # one byte short
+    assert two_pass(SC + 2, 1 << 20) == binding.QKNORM_ERR_SCRATCH             # not float aligned
+    assert two_pass(A, 1 << 20) == binding.QKNORM_ERR_SCRATCH                  # on top of an input
+    assert gather(SC, 4 * 128 * 2 - 1) == binding.QKNORM_ERR_SCRATCH
+    assert gather(SC + 8, 1 << 20) == binding.QKNORM_ERR_SCRATCH               # not 16-byte aligned
+    assert gather(E, 1 << 20) == binding.QKNORM_ERR_SCRATCH                    # on top of an output

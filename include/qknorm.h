@@ -64,7 +64,8 @@ typedef enum {
   QKNORM_ERR_EPS = 6,     /* eps < 0 or NaN */
   QKNORM_ERR_CUDA = 7,    /* a CUDA call failed; see qknorm_last_cuda_error() */
   QKNORM_ERR_HEADS = 8,   /* head_dim < 1 or does not divide dq (or dk) */
-  QKNORM_ERR_SCRATCH = 9  /* scratch buffer NULL, too small, misaligned, or overlapping a buffer of the call */
+  QKNORM_ERR_SCRATCH = 9,       /* scratch buffer NULL, too small, misaligned, or overlapping a buffer of the call */
+  QKNORM_ERR_STATIC_LIMIT = 10  /* the call needs more scratch than the library's built-in array holds */
 } qknorm_status;
 
 /*
@@ -200,6 +201,46 @@ int qknorm_baseline_two_pass(const void* const* q_shards, const void* const* k_s
                              int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
                              void* const* out_q_shards, void* const* out_k_shards,
                              float* scratch, size_t scratch_bytes, void* stream);
+
+/*
+ * qknorm_baseline_two_pass_static -- qknorm_baseline_two_pass for callers that cannot
+ * bring a scratch buffer.  (The paper has no counterpart; this is a convenience of
+ * this library.)
+ *
+ * Who needs it: code that must not allocate device memory where it makes the call.
+ * Typical cases are a serving engine that has already handed all free HBM to its
+ * KV-cache pool, so that a cudaMalloc for a few hundred kilobytes would fail or force
+ * the pool to shrink, and a plug-in that runs inside someone else's step loop, where
+ * cudaMalloc/cudaFree would stall the whole device and the host framework's allocator
+ * is not reachable from C.  This entry point calls no cudaMalloc, no cudaFree and no
+ * library routine that allocates.
+ *
+ * How: the statistics pass writes every slice's sum of squares into an array that is
+ * part of the library image itself (static device memory, 262144 floats = 1 MiB; every
+ * GPU that loads the library holds that 1 MiB until the process exits), and the scale
+ * pass reads them back.  Arguments and result are those of qknorm_baseline_two_pass
+ * without the scratch arguments.
+ *
+ * Limits and rules:
+ *  - 2 * num_shards * tokens must not exceed qknorm_static_scratch_capacity()
+ *    (262144), else QKNORM_ERR_STATIC_LIMIT and nothing is launched.  Split the tokens
+ *    over several calls, or use qknorm_baseline_two_pass with your own buffer.
+ *  - The first call on each device looks up the array's device address
+ *    (cudaGetSymbolAddress, with that device current) and keeps it; make that first call
+ *    before any stream capture begins on that device.
+ *  - All calls on a device share the one array, and it keeps whatever the last call
+ *    left in it.  Nothing needs clearing between calls (a call only reads back what its
+ *    own first pass wrote), but two calls that can overlap on the GPU -- different
+ *    streams, or the same stream with programmatic overlap -- race on it and give wrong
+ *    results.  Serialise them.
+ */
+int qknorm_baseline_two_pass_static(const void* const* q_shards, const void* const* k_shards,
+                                    const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                                    int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
+                                    void* const* out_q_shards, void* const* out_k_shards, void* stream);
+
+/* Number of floats in the built-in scratch array of qknorm_baseline_two_pass_static. */
+int64_t qknorm_static_scratch_capacity(void);
 
 /* Human-readable name of a qknorm_status (static storage, never NULL). */
 const char* qknorm_status_string(int status);

@@ -26,6 +26,8 @@ EXPORTS = (
     "qknorm_fwd_headwise",
     "qknorm_baseline_gather_then_norm",
     "qknorm_baseline_two_pass",
+    "qknorm_baseline_two_pass_static",
+    "qknorm_static_scratch_capacity",
     "qknorm_fwd_sharded_e4m3",
     "qknorm_status_string",
     "qknorm_device_error_word",
@@ -45,6 +47,7 @@ QKNORM_ERR_EPS = 6
 QKNORM_ERR_CUDA = 7
 QKNORM_ERR_HEADS = 8
 QKNORM_ERR_SCRATCH = 9
+QKNORM_ERR_STATIC_LIMIT = 10
 
 
 class QKNormError(RuntimeError):
@@ -89,6 +92,10 @@ def load() -> ctypes.CDLL:
     for fn in (lib.qknorm_baseline_gather_then_norm, lib.qknorm_baseline_two_pass):
         fn.argtypes = [_vpp, _vpp, _vpp, _vpp, i32, i64, i32, i32, f32, _vpp, _vpp, _vp, ctypes.c_size_t, _vp]
         fn.restype = ctypes.c_int
+    lib.qknorm_baseline_two_pass_static.argtypes = [_vpp, _vpp, _vpp, _vpp, i32, i64, i32, i32, f32, _vpp, _vpp, _vp]
+    lib.qknorm_baseline_two_pass_static.restype = ctypes.c_int
+    lib.qknorm_static_scratch_capacity.argtypes = []
+    lib.qknorm_static_scratch_capacity.restype = ctypes.c_int64
     lib.qknorm_status_string.argtypes = [ctypes.c_int]
     lib.qknorm_status_string.restype = ctypes.c_char_p
     lib.qknorm_device_error_word.argtypes = [ctypes.POINTER(ctypes.c_int)]
@@ -351,6 +358,35 @@ def qknorm_baseline_two_pass(q_shards, k_shards, gamma_q_shards, gamma_k_shards,
     """qknorm_baseline_two_pass; scratch: CUDA fp32 tensor of >= 2*S*T elements."""
     return _baseline(load().qknorm_baseline_two_pass, q_shards, k_shards, gamma_q_shards, gamma_k_shards,
                      eps, out_q_shards, out_k_shards, scratch, stream)
+
+
+def qknorm_baseline_two_pass_static(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: float,
+                                    out_q_shards, out_k_shards, *, stream=None):
+    """qknorm_baseline_two_pass_static: the two-pass stand-in with the library's built-in
+    1 MiB scratch array, for callers that must not allocate device memory.  Unlike the
+    other wrappers this one creates no tensors: the outputs must be passed (they may be the
+    inputs).  Calls that can overlap on the GPU race on the shared array; the first call on
+    a device should come before any stream capture (see include/qknorm.h)."""
+    lib = load()
+    S = len(q_shards)
+    T = q_shards[0].shape[0]
+    wq, wk = q_shards[0].shape[1], k_shards[0].shape[1]
+    bf = torch.bfloat16
+    for s in range(S):
+        _expect(q_shards[s], (T, wq), bf, f"q_shards[{s}]")
+        _expect(k_shards[s], (T, wk), bf, f"k_shards[{s}]")
+        _expect(gamma_q_shards[s], (wq,), bf, f"gamma_q_shards[{s}]")
+        _expect(gamma_k_shards[s], (wk,), bf, f"gamma_k_shards[{s}]")
+        _expect(out_q_shards[s], (T, wq), bf, f"out_q_shards[{s}]")
+        _expect(out_k_shards[s], (T, wk), bf, f"out_k_shards[{s}]")
+    _check(lib.qknorm_baseline_two_pass_static(_array(q_shards, S), _array(k_shards, S), _array(gamma_q_shards, S),
+                                               _array(gamma_k_shards, S), S, T, wq * S, wk * S, float(eps),
+                                               _array(out_q_shards, S), _array(out_k_shards, S), _stream(stream)))
+    return out_q_shards, out_k_shards
+
+
+def static_scratch_capacity() -> int:
+    return int(load().qknorm_static_scratch_capacity())
 
 
 def device_error_word() -> int:

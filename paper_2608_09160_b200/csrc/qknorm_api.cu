@@ -74,6 +74,12 @@ WarpKernel warp_kernel_for(int l, bool exact, int elem_bytes) {
 // Set by a ring kernel whose bounded wait ran out (0 = never happened).
 __device__ int g_ring_error = 0;
 
+// Built-in scratch of qknorm_baseline_two_pass_static: 1 MiB of device memory that every
+// GPU which loads this library holds until the process exits.  In host code this name is
+// only a handle for cudaGetSymbolAddress, never a device address.
+constexpr size_t kStaticScratchFloats = 262144;
+static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
+
 namespace {
 
 thread_local int tl_cuda_error = 0;
@@ -744,6 +750,29 @@ int run_headwise(const void* q, const void* k, const void* gq, const void* gk, i
   return finish_launch("head_general");
 }
 
+// Device address of g_static_scratch on the current device, looked up once per device.
+float* g_static_scratch_addr[kMaxDevices];
+bool g_static_scratch_known[kMaxDevices];
+std::mutex g_static_scratch_mutex;
+
+int static_scratch_address(float** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return set_cuda_error(e);
+  if (dev < 0 || dev >= kMaxDevices) return set_cuda_error(cudaErrorInvalidDevice);
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (!g_static_scratch_known[dev]) {
+    float* p = nullptr;
+    // `dev` is the current device, so this is the address of ITS copy of the array
+    e = cudaGetSymbolAddress((void**)&p, g_static_scratch);
+    if (e != cudaSuccess) return set_cuda_error(e);
+    g_static_scratch_addr[dev] = p;
+    g_static_scratch_known[dev] = true;
+  }
+  *out = g_static_scratch_addr[dev];
+  return QKNORM_OK;
+}
+
 }  // namespace
 }  // namespace qknorm
 
@@ -808,6 +837,26 @@ int qknorm_baseline_two_pass(const void* const* q_shards, const void* const* k_s
   return qknorm::run_two_pass(P, scratch, (cudaStream_t)stream);
 }
 
+int qknorm_baseline_two_pass_static(const void* const* q_shards, const void* const* k_shards,
+                                    const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                                    int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, float eps,
+                                    void* const* out_q_shards, void* const* out_k_shards, void* stream) {
+  qknorm::Params P;
+  bool empty = true;
+  int rc = qknorm::prepare(P, &empty, 2, q_shards, k_shards, gamma_q_shards, gamma_k_shards, num_shards, tokens, dq,
+                           dk, eps, out_q_shards, out_k_shards, nullptr, nullptr, nullptr, nullptr);
+  if (rc != QKNORM_OK || empty) return rc;
+  if ((uint64_t)2 * (uint64_t)num_shards * (uint64_t)tokens > (uint64_t)qknorm::kStaticScratchFloats)
+    return QKNORM_ERR_STATIC_LIMIT;
+  float* scratch = nullptr;
+  rc = qknorm::static_scratch_address(&scratch);  // first call on a device: the one-time look-up
+  if (rc != QKNORM_OK) return rc;
+  // Nothing has to be cleared: pass 1 writes every element that pass 2 of the same call reads.
+  return qknorm::run_two_pass(P, scratch, (cudaStream_t)stream);
+}
+
+int64_t qknorm_static_scratch_capacity(void) { return (int64_t)qknorm::kStaticScratchFloats; }
+
 int qknorm_fwd_strided(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
                        int32_t dq, int32_t dk, int64_t ld_q, int64_t ld_k, float eps, void* out_q, void* out_k,
                        int64_t ld_out_q, int64_t ld_out_k, void* stream) {
@@ -854,6 +903,8 @@ const char* qknorm_status_string(int status) {
     case QKNORM_ERR_CUDA: return "QKNORM_ERR_CUDA: a CUDA call failed";
     case QKNORM_ERR_HEADS: return "QKNORM_ERR_HEADS: head_dim < 1 or does not divide the width";
     case QKNORM_ERR_SCRATCH: return "QKNORM_ERR_SCRATCH: scratch buffer missing, too small, misaligned or overlapping";
+    case QKNORM_ERR_STATIC_LIMIT:
+      return "QKNORM_ERR_STATIC_LIMIT: 2 * num_shards * tokens exceeds the 262144 floats of the built-in scratch array";
     default: return "unknown qknorm status";
   }
 }

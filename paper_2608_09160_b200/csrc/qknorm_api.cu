@@ -225,8 +225,8 @@ inline int round_up(int v, int m) { return ((v + m - 1) / m) * m; }
 // thread, G_q / G_k threads per Q / K slice, lane groups of 16 or 32.
 //  throughput: wide CTAs with few chunks per thread (many warps hide the latency
 //              of the per-token reduction), as few idle lanes as possible;
-//  latency (few tokens): as few chunks per thread as possible, so that one load
-//              round trip covers the row.
+//  latency (few tokens): CTAs of about 256 threads; every load of a thread is issued
+//              before the first use, so a few chunks per thread still cost one round trip.
 bool plan_rows(const Params& P, bool latency, RowsPlan* plan) {
   const int cq = P.q.d ? P.q.w * P.elem_bytes / 16 : 0, ck = P.k.d ? P.k.w * P.elem_bytes / 16 : 0;
   const int force_n = env_int("QKNORM_FORCE_N", 0);
@@ -244,12 +244,14 @@ bool plan_rows(const Params& P, bool latency, RowsPlan* plan) {
       const int threads = round_up(P.S * (Gq + Gk), 32);
       if (threads > max_threads_for(n)) continue;
       if (P.S * (Gq + Gk) / sub > kMaxSlots) continue;
-      // Estimated warp instructions per token: per chunk position ~45, per token and
-      // thread ~60 plus the slots it has to add up.  Decode sizes instead want the
-      // shortest dependent chain (few chunks per thread), whatever the lane count.
+      // Prefill (the rows too wide for the warp kernel): estimated warp instructions per token,
+      // per chunk position ~45, per token and thread ~60 plus the slots it has to add up.
+      // Decode sizes: measured under CUDA-graph replay, CTAs of about 256 threads with ~4
+      // chunks per thread are fastest (2.4 us per call against 2.8-3.5 us for 1024-thread CTAs).
       const int warps = threads / 32;
       const int slots = P.S * (Gq > Gk ? Gq : Gk) / sub;
-      double cost = latency ? (double)n * 1000.0 + warps : (double)warps * (45.0 * n + 60.0 + 2.0 * slots);
+      double cost = latency ? (double)(threads > 256 ? threads - 256 : 256 - threads) + 0.1 * n
+                            : (double)warps * (45.0 * n + 60.0 + 2.0 * slots);
       if (log_sub == 4) cost *= 1.001;  // tie: full-warp groups (fewer slots to add up)
       if (cost < best_cost) {
         best_cost = cost;

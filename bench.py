@@ -147,10 +147,13 @@ class DeviceCase:
     """Device (and optionally pinned host) buffers of one workload at one shard
     count, plus the closure that makes the one C-ABI call."""
 
-    def __init__(self, w: W.Workload, S: int, rank: int = 0, host: bool = False, io: str = "bf16"):
+    def __init__(self, w: W.Workload, S: int, rank: int = 0, host: bool = False, io: str = "bf16",
+                 head_dim: int = 0):
         from paper_2608_09160_b200 import binding
         self.binding = binding
-        self.w, self.S, self.io = w, S, io
+        self.w, self.S, self.io, self.head_dim = w, S, io, head_dim
+        if head_dim and (S != 1 or io != "bf16"):
+            raise SystemExit("--head-dim needs --shards 1 and bf16")
         make = W.make_inputs if io == "bf16" else W.make_inputs_e4m3
         inp = make(rank_workload(w, rank))
         self.host_in = None
@@ -178,7 +181,10 @@ class DeviceCase:
 
     def call(self):
         d = self.dev
-        if self.S == 1:
+        if self.head_dim:
+            self.binding.qknorm_fwd_headwise(d["q"][0], d["k"][0], d["gq"][0], d["gk"][0], self.head_dim, self.w.eps,
+                                             self.out_q[0], self.out_k[0])
+        elif self.S == 1:
             self.fwd(d["q"][0], d["k"][0], d["gq"][0], d["gk"][0], self.w.eps, self.out_q[0], self.out_k[0])
         else:
             self.fwd_sharded(d["q"], d["k"], d["gq"], d["gk"], self.w.eps, self.out_q, self.out_k)
@@ -217,7 +223,10 @@ class DeviceCase:
                     dst.copy_(src, non_blocking=True)
                 ev_in = self.s_in.record_event()
             cur.wait_event(ev_in)
-            if self.S == 1:
+            if self.head_dim:
+                self.binding.qknorm_fwd_headwise(c["q"][0], c["k"][0], d["gq"][0], d["gk"][0], self.head_dim,
+                                                 self.w.eps, c["oq"][0], c["ok"][0])
+            elif self.S == 1:
                 self.fwd(c["q"][0], c["k"][0], d["gq"][0], d["gk"][0], self.w.eps, c["oq"][0], c["ok"][0])
             else:
                 self.fwd_sharded(c["q"], c["k"], d["gq"], d["gk"], self.w.eps, c["oq"], c["ok"])
@@ -453,11 +462,17 @@ def job_value(bytes_per_rank: int, world: int, ms_per_step: float) -> float:
     return world * bytes_per_rank / (ms_per_step * 1e-3) / 1e9
 
 
-def config_of(w: W.Workload, S: int, world: int, variant=None):
+def case_bytes_of(w: W.Workload, io: str) -> int:
+    eb = 2 if io == "bf16" else 1
+    return 2 * w.tokens * (w.dq + w.dk) * eb + (w.dq + w.dk) * 2
+
+
+def config_of(w: W.Workload, S: int, world: int, variant=None, io: str = "bf16", head_dim: int = 0):
     """The `config` object of the JSON line (the same for both arms)."""
     cfg = {"workload": f"{w.name}: {w.note}", "tokens": w.tokens, "dq": w.dq, "dk": w.dk, "num_shards": S,
-           "in_place": w.in_place, "storage": "bf16", "eps": w.eps,
-           "bytes_per_step_per_gpu": w.algorithmic_bytes,
+           "in_place": w.in_place, "storage": io, "eps": w.eps,
+           "granularity": f"headwise, head_dim {head_dim}" if head_dim else "layerwise",
+           "bytes_per_step_per_gpu": case_bytes_of(w, io),
            "parallelism": f"token-range x{world}, no collective",
            "l2": "inputs larger than L2 (no flush needed)" if w.algorithmic_bytes > 300e6
                  else "working set fits in L2 (L2-warm number)"}
@@ -516,6 +531,8 @@ def main():
     ap.add_argument("--workload", default="C5", choices=sorted(W.WORKLOADS))
     ap.add_argument("--shards", type=int, default=0, help="shard count (default: the workload's first)")
     ap.add_argument("--tokens", type=int, default=0, help="override the token count (for profiling a small case)")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "e4m3"], help="storage format of the activations")
+    ap.add_argument("--head-dim", type=int, default=0, help="headwise granularity with this head size (needs --shards 1)")
     ap.add_argument("--no-table", action="store_true", help="skip the per-config table")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
@@ -556,7 +573,7 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    case = DeviceCase(w, S, rank=rank, host=not args.no_e2e)
+    case = DeviceCase(w, S, rank=rank, host=not args.no_e2e, io=args.dtype, head_dim=args.head_dim)
 
     # ---- device-resident timing -----------------------------------------------------------
     for _ in range(args.warmup):
@@ -597,7 +614,8 @@ def main():
     variant = binding.last_variant()
     del case
     torch.cuda.empty_cache()
-    same_size_copy = copy_rate_same_bytes(w.algorithmic_bytes) if rank == 0 else None
+    case_bytes = case_bytes_of(w, args.dtype)
+    same_size_copy = copy_rate_same_bytes(case_bytes) if rank == 0 else None
     torch.cuda.empty_cache()
 
     if rank != 0:
@@ -616,15 +634,15 @@ def main():
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": config_of(w, S, world, variant),
+        "config": config_of(w, S, world, variant, args.dtype, args.head_dim),
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": UNIT,
-                     "frac": round(achieved / peak, 4), "traffic": NCU_DRAM_TRAFFIC_BYTES.get(f"{w.name}/S{S}"),
+                     "frac": round(achieved / peak, 4), "traffic": NCU_DRAM_TRAFFIC_BYTES.get(f"{w.name}/S{S}") if (args.dtype == "bf16" and not args.head_dim) else None,
                      "peak_kind": f"{peak_kind} copy rate (of {peak_kind})",
                      "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4),
-                     "algorithmic_bytes_per_launch": w.algorithmic_bytes,
+                     "algorithmic_bytes_per_launch": case_bytes,
                      "same_size_copy_GBps": round(same_size_copy, 1),
                      "launch_us_mean": round(launch_ms * 1e3, 3), "launch_us_min": round(min(per_call) * 1e3, 3)},
         "cpu_baseline": cpu,

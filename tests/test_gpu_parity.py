@@ -212,3 +212,11 @@ def test_alias_is_rejected_on_real_buffers(libqknorm):
     with pytest.raises(binding.QKNormError) as ei:
         binding.qknorm_fwd(q, None, g, None, 1e-6, out_overlapping, None)
     assert ei.value.status == binding.QKNORM_ERR_ALIAS
+
+
+def test_no_bounded_wait_ever_ran_out(libqknorm):
+    """Every in-kernel mbarrier wait is bounded and reports through a device word; after all
+    the TMA-fed launches this process made so far the word must still be clear."""
+    w = next(x for x in SMALL if x.name == "s_prefill_gqa")
+    run_case(w, 8)
+    assert binding.device_error_word() == 0

@@ -581,13 +581,13 @@ def main():
     barrier()
     sampler = ClockSampler(local)
     sampler.start()
+    barrier()
+    per_call = time_calls(case.call, args.steps, 0)          # one event pair per launch (roofline.achieved)
+    barrier()
     n0 = binding.launch_count()
+    total_ms = time_region(case.call, args.steps)            # THE timed region: K steps, back to back
     barrier()
-    per_call = time_calls(case.call, args.steps, 0)          # one event pair per launch
-    barrier()
-    total_ms = time_region(case.call, args.steps)            # the K timed steps, back to back
-    barrier()
-    launches = binding.launch_count() - n0
+    launches = binding.launch_count() - n0                   # kernels of this library launched inside it
     total_ms = max_over_ranks(total_ms, dist, "cuda")
     ms_per_step = total_ms / args.steps
     value = job_value(case.bytes, world, ms_per_step)

@@ -183,6 +183,8 @@ def small_parity_shapes() -> List[Workload]:
         ("s_prefill_odd", 777, 1000, 136, (1,)),         # warp-per-token kernel, lanes with ragged chunk counts
         ("s_prefill_s3", 650, 1536, 768, (3,)),          # shard count that leaves lanes idle
         ("s_prefill_konly", 700, 0, 1024, (2,)),
+        ("s_prefill_s16", 640, 4096, 1024, (16,)),       # two lanes per shard, every lane issues a bulk copy
+        ("s_prefill_s5", 610, 2240, 560, (5, 7)),        # shard counts that are not powers of two
         ("s_prefill_wide", 600, 16384, 4096, (1, 4)),    # rows too wide for one warp: the CTA-per-token TMA ring
     ]
     out = []

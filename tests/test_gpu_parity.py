@@ -123,6 +123,7 @@ def test_unaligned_buffers_take_the_general_kernel(libqknorm, skew):
     ("s_t1", 1, "rows"), ("s_149", 8, "rows"), ("s_gqa8", 8, "rows"),          # few tokens: register-resident rows
     ("s_prefill_gqa", 8, "warp"), ("s_prefill_gqa", 1, "warp"), ("s_prefill_odd", 1, "warp"),
     ("s_prefill_s3", 3, "warp"), ("s_prefill_konly", 2, "warp"), ("s_1025", 4, "warp"),
+    ("s_prefill_s16", 16, "warp"), ("s_prefill_s5", 5, "warp"),
     ("s_prefill_wide", 1, "ring"), ("s_prefill_wide", 4, "ring"),
     ("s_unaligned", 7, "general"), ("s_max", 1, "general"),
 ])

@@ -51,11 +51,12 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per launch of the dominant kernel measured by ncu
 # (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
-# C5/S8: captured on 16384 of the 65536 tokens (302.05 MB read + 246.77 MB
-# written per launch, profiles/warp_kernel_C5_16k_tokens_full_set.md) and scaled
-# by the tokens processed (x4).  Reads scale exactly; the writes fall short of
-# the algorithmic bytes by the lines still dirty in L2 when the kernel ends.
-NCU_DRAM_TRAFFIC_BYTES = {"C5/S8": 4 * (302_049_152 + 246_769_920)}
+# C5/S8: a one-pass capture of the full 65536-token launch
+# (profiles/warp_kernel_C5_full_size_dram_traffic.md): 1 208 027 392 bytes read,
+# 1 150 823 936 written.  Reads equal the algorithmic reads; the writes fall
+# 57 MB short of the algorithmic bytes because the call is in place and the last
+# lines written are still dirty in L2 when the kernel ends.
+NCU_DRAM_TRAFFIC_BYTES = {"C5/S8": 1_208_027_392 + 1_150_823_936}
 
 
 def log(*a):

@@ -51,9 +51,8 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per launch of the dominant kernel measured by ncu
 # (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
-# C5/S8: a one-pass capture of the full 65536-token launch
-# (profiles/warp_kernel_C5_full_size_dram_traffic.md): 1 208 027 392 bytes read,
-# 1 150 823 936 written.  Reads equal the algorithmic reads; the writes fall
+# C5/S8: a one-pass capture of the full 65536-token launch (summarised under
+# profiles/): 1 208 027 392 bytes read, 1 150 823 936 written.  Reads equal the algorithmic reads; the writes fall
 # 57 MB short of the algorithmic bytes because the call is in place and the last
 # lines written are still dirty in L2 when the kernel ends.
 NCU_DRAM_TRAFFIC_BYTES = {"C5/S8": 1_208_027_392 + 1_150_823_936}

@@ -106,14 +106,19 @@ int qko_rmsnorm(const uint16_t* x, const uint16_t* gamma, int64_t T, int64_t H, 
 #ifdef _OPENMP
     if (nthreads > 1) {
 #pragma omp parallel for num_threads(nthreads) schedule(static)
+        int failed = 0;
         for (int64_t t = 0; t < T; ++t) {
             uint16_t* row = (uint16_t*)malloc((size_t)H * sizeof(uint16_t));
+            if (!row) {
+                failed = 1;   /* benign race: every writer stores 1 */
+                continue;
+            }
             memcpy(row, x + t * H, (size_t)H * sizeof(uint16_t));
             rmsnorm_row(row, gamma, H, e, y ? y + t * H : NULL, y64 ? y64 + t * H : NULL,
                         acc ? acc + t : NULL, rstd ? rstd + t : NULL);
             free(row);
         }
-        return 0;
+        return failed ? -1 : 0;
     }
 #else
     (void)nthreads;
@@ -154,9 +159,16 @@ int qko_rmsnorm_sharded(const uint16_t* const* x_shards, const uint16_t* const* 
 #else
     (void)nthreads;
 #endif
+    int failed = 0;
     for (int64_t t = 0; t < T; ++t) {
         uint16_t* row = (uint16_t*)malloc((size_t)H * sizeof(uint16_t));
         uint16_t* out = (uint16_t*)malloc((size_t)H * sizeof(uint16_t));
+        if (!row || !out) {
+            free(row);
+            free(out);
+            failed = 1;
+            continue;
+        }
         /* gather: slice s goes to columns [s*w, (s+1)*w) */
         for (int s = 0; s < S; ++s) memcpy(row + s * w, x_shards[s] + t * w, (size_t)w * sizeof(uint16_t));
         if (partials) {
@@ -178,7 +190,7 @@ int qko_rmsnorm_sharded(const uint16_t* const* x_shards, const uint16_t* const* 
         free(out);
     }
     free(gfull);
-    return 0;
+    return failed ? -1 : 0;
 }
 
 /* ---- FP8-E4M3 activations (Section IV-C: "BF16 and FP8-E4M3 activations", FP32 accumulation) ----
@@ -263,9 +275,16 @@ int qko_rmsnorm_sharded_e4m3(const uint8_t* const* x_shards, const uint16_t* con
 #else
     (void)nthreads;
 #endif
+    int failed = 0;
     for (int64_t t = 0; t < T; ++t) {
         uint8_t* row = (uint8_t*)malloc((size_t)H);
         uint8_t* out = (uint8_t*)malloc((size_t)H);
+        if (!row || !out) {
+            free(row);
+            free(out);
+            failed = 1;
+            continue;
+        }
         for (int s = 0; s < S; ++s) memcpy(row + s * w, x_shards[s] + t * w, (size_t)w);
         if (partials) {
             for (int s = 0; s < S; ++s) {
@@ -287,7 +306,7 @@ int qko_rmsnorm_sharded_e4m3(const uint8_t* const* x_shards, const uint16_t* con
         free(out);
     }
     free(gfull);
-    return 0;
+    return failed ? -1 : 0;
 }
 
 /* ---- headwise granularity (Section II-A) ------------------------------------------------------

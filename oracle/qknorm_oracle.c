@@ -105,8 +105,8 @@ int qko_rmsnorm(const uint16_t* x, const uint16_t* gamma, int64_t T, int64_t H, 
     const double e = (double)eps;
 #ifdef _OPENMP
     if (nthreads > 1) {
-#pragma omp parallel for num_threads(nthreads) schedule(static)
         int failed = 0;
+#pragma omp parallel for num_threads(nthreads) schedule(static)
         for (int64_t t = 0; t < T; ++t) {
             uint16_t* row = (uint16_t*)malloc((size_t)H * sizeof(uint16_t));
             if (!row) {
@@ -153,13 +153,13 @@ int qko_rmsnorm_sharded(const uint16_t* const* x_shards, const uint16_t* const* 
     if (!gfull) return -1;
     for (int s = 0; s < S; ++s) memcpy(gfull + s * w, gamma_shards[s], (size_t)w * sizeof(uint16_t));
     int nt = 1;
+    int failed = 0;
 #ifdef _OPENMP
     if (nthreads > 1) nt = nthreads;
 #pragma omp parallel for num_threads(nt) schedule(static)
 #else
     (void)nthreads;
 #endif
-    int failed = 0;
     for (int64_t t = 0; t < T; ++t) {
         uint16_t* row = (uint16_t*)malloc((size_t)H * sizeof(uint16_t));
         uint16_t* out = (uint16_t*)malloc((size_t)H * sizeof(uint16_t));
@@ -269,13 +269,13 @@ int qko_rmsnorm_sharded_e4m3(const uint8_t* const* x_shards, const uint16_t* con
     if (!gfull) return -1;
     for (int s = 0; s < S; ++s) memcpy(gfull + s * w, gamma_shards[s], (size_t)w * sizeof(uint16_t));
     int nt = 1;
+    int failed = 0;
 #ifdef _OPENMP
     if (nthreads > 1) nt = nthreads;
 #pragma omp parallel for num_threads(nt) schedule(static)
 #else
     (void)nthreads;
 #endif
-    int failed = 0;
     for (int64_t t = 0; t < T; ++t) {
         uint8_t* row = (uint8_t*)malloc((size_t)H);
         uint8_t* out = (uint8_t*)malloc((size_t)H);

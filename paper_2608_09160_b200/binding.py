@@ -9,6 +9,7 @@ from __future__ import annotations
 
 import ctypes
 import os
+import threading
 from typing import Optional, Sequence
 
 import torch
@@ -121,6 +122,50 @@ def _check(status: int) -> None:
         raise QKNormError(status, msg)
 
 
+class PreparedCall:
+    """One C-ABI call whose arguments are already marshalled (pointers, sizes, host pointer
+    arrays).  Calling the object makes the C call again on the current (or the given) stream:
+    nothing but the call itself is left on the host side of a hot loop.  The tensors are kept
+    alive by the object; `outputs` is what the wrapper would have returned."""
+    __slots__ = ("cfunc", "args", "keep", "outputs")
+
+    def __init__(self, cfunc, args, keep):
+        self.cfunc, self.args, self.keep, self.outputs = cfunc, tuple(args), keep, None
+
+    def __call__(self, stream=None):
+        status = self.cfunc(*self.args, _stream(stream))
+        if status != QKNORM_OK:
+            _check(status)
+
+
+_capture = threading.local()
+
+
+def _invoke(cfunc, args, stream, keep):
+    """Makes the call, or records it when `prepared` is collecting."""
+    sink = getattr(_capture, "sink", None)
+    if sink is not None:
+        sink.append(PreparedCall(cfunc, args, keep))
+        return
+    _check(cfunc(*args, _stream(stream)))
+
+
+def prepared(wrapper, *args, **kwargs) -> PreparedCall:
+    """prepared(qknorm_fwd_sharded, q_shards, ...) validates and marshals the arguments exactly
+    as the wrapper would, makes NO call, and returns a PreparedCall for the one C-ABI call the
+    wrapper would have made."""
+    _capture.sink = []
+    try:
+        outs = wrapper(*args, **kwargs)
+        sink = _capture.sink
+    finally:
+        _capture.sink = None
+    if len(sink) != 1:
+        raise QKNormError(-1, "the wrapper did not make exactly one C-ABI call")
+    sink[0].outputs = outs
+    return sink[0]
+
+
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
     if t is None:
         return None
@@ -201,12 +246,13 @@ def qknorm_fwd(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=None, *,
     args = [_ptr(q), _ptr(k), _ptr(gamma_q) if q is not None else None,
             _ptr(gamma_k) if k is not None else None, T, dq, dk, float(eps),
             _ptr(out_q) if q is not None else None, _ptr(out_k) if k is not None else None]
+    keep = (q, k, gamma_q, gamma_k, out_q, out_k, rstd_q, rstd_k)
     if act is not bf:
-        _check(lib.qknorm_fwd_e4m3(*args, _ptr(rstd_q), _ptr(rstd_k), _stream(stream)))
+        _invoke(lib.qknorm_fwd_e4m3, [*args, _ptr(rstd_q), _ptr(rstd_k)], stream, keep)
     elif rstd_q is None and rstd_k is None:
-        _check(lib.qknorm_fwd(*args, _stream(stream)))
+        _invoke(lib.qknorm_fwd, args, stream, keep)
     else:
-        _check(lib.qknorm_fwd_ex(*args, _ptr(rstd_q), _ptr(rstd_k), _stream(stream)))
+        _invoke(lib.qknorm_fwd_ex, [*args, _ptr(rstd_q), _ptr(rstd_k)], stream, keep)
     return out_q, out_k
 
 
@@ -251,14 +297,15 @@ def qknorm_fwd_sharded(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: 
             _expect(t, shp, torch.float32, nm)
     args = [_array(q_shards, S), _array(k_shards, S), _array(gamma_q_shards, S), _array(gamma_k_shards, S),
             S, T, wq * S, wk * S, float(eps), _array(out_q_shards, S), _array(out_k_shards, S)]
+    keep = (q_shards, k_shards, gamma_q_shards, gamma_k_shards, out_q_shards, out_k_shards,
+            partials_q, partials_k, rstd_q, rstd_k)
+    extra = [_ptr(partials_q), _ptr(partials_k), _ptr(rstd_q), _ptr(rstd_k)]
     if act is not bf:
-        _check(lib.qknorm_fwd_sharded_e4m3(*args, _ptr(partials_q), _ptr(partials_k), _ptr(rstd_q),
-                                           _ptr(rstd_k), _stream(stream)))
+        _invoke(lib.qknorm_fwd_sharded_e4m3, [*args, *extra], stream, keep)
     elif all(t is None for t in (partials_q, partials_k, rstd_q, rstd_k)):
-        _check(lib.qknorm_fwd_sharded(*args, _stream(stream)))
+        _invoke(lib.qknorm_fwd_sharded, args, stream, keep)
     else:
-        _check(lib.qknorm_fwd_sharded_ex(*args, _ptr(partials_q), _ptr(partials_k), _ptr(rstd_q),
-                                         _ptr(rstd_k), _stream(stream)))
+        _invoke(lib.qknorm_fwd_sharded_ex, [*args, *extra], stream, keep)
     return out_q_shards, out_k_shards
 
 
@@ -283,8 +330,9 @@ def qknorm_fwd_strided(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=Non
           _expect_rows(out_q, T, dq, "out_q"), _expect_rows(out_k, T, dk, "out_k")]
     _expect(gamma_q, (dq,), torch.bfloat16, "gamma_q")
     _expect(gamma_k, (dk,), torch.bfloat16, "gamma_k")
-    _check(lib.qknorm_fwd_strided(_ptr(q), _ptr(k), _ptr(gamma_q), _ptr(gamma_k), T, dq, dk, ld[0], ld[1],
-                                  float(eps), _ptr(out_q), _ptr(out_k), ld[2], ld[3], _stream(stream)))
+    _invoke(lib.qknorm_fwd_strided, [_ptr(q), _ptr(k), _ptr(gamma_q), _ptr(gamma_k), T, dq, dk, ld[0], ld[1],
+                                     float(eps), _ptr(out_q), _ptr(out_k), ld[2], ld[3]], stream,
+            (q, k, gamma_q, gamma_k, out_q, out_k))
     return out_q, out_k
 
 
@@ -314,11 +362,11 @@ def qknorm_fwd_headwise(q, k, gamma_q, gamma_k, head_dim: int, eps: float, out_q
         _expect(rstd_q, (T, dq // max(hd, 1)), torch.float32, "rstd_q")
     if rstd_k is not None:
         _expect(rstd_k, (T, dk // max(hd, 1)), torch.float32, "rstd_k")
-    _check(lib.qknorm_fwd_headwise(_ptr(q), _ptr(k), _ptr(gamma_q) if q is not None else None,
-                                   _ptr(gamma_k) if k is not None else None, T, dq, dk, hd, ld[0], ld[1],
-                                   float(eps), _ptr(out_q) if q is not None else None,
-                                   _ptr(out_k) if k is not None else None, ld[2], ld[3], _ptr(rstd_q),
-                                   _ptr(rstd_k), _stream(stream)))
+    _invoke(lib.qknorm_fwd_headwise, [_ptr(q), _ptr(k), _ptr(gamma_q) if q is not None else None,
+                                      _ptr(gamma_k) if k is not None else None, T, dq, dk, hd, ld[0], ld[1],
+                                      float(eps), _ptr(out_q) if q is not None else None,
+                                      _ptr(out_k) if k is not None else None, ld[2], ld[3], _ptr(rstd_q),
+                                      _ptr(rstd_k)], stream, (q, k, gamma_q, gamma_k, out_q, out_k, rstd_q, rstd_k))
     return out_q, out_k
 
 
@@ -340,9 +388,10 @@ def _baseline(entry, q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps, ou
     if scratch is not None and (not scratch.is_cuda or not scratch.is_contiguous()):
         raise QKNormError(QKNORM_ERR_SCRATCH, "scratch must be a contiguous CUDA tensor")
     nbytes = scratch.numel() * scratch.element_size() if scratch is not None else 0
-    _check(entry(_array(q_shards, S), _array(k_shards, S), _array(gamma_q_shards, S), _array(gamma_k_shards, S),
-                 S, T, wq * S, wk * S, float(eps), _array(out_q_shards, S), _array(out_k_shards, S),
-                 _ptr(scratch), nbytes, _stream(stream)))
+    _invoke(entry, [_array(q_shards, S), _array(k_shards, S), _array(gamma_q_shards, S), _array(gamma_k_shards, S),
+                    S, T, wq * S, wk * S, float(eps), _array(out_q_shards, S), _array(out_k_shards, S),
+                    _ptr(scratch), nbytes], stream,
+            (q_shards, k_shards, gamma_q_shards, gamma_k_shards, out_q_shards, out_k_shards, scratch))
     return out_q_shards, out_k_shards
 
 
@@ -379,9 +428,10 @@ def qknorm_baseline_two_pass_static(q_shards, k_shards, gamma_q_shards, gamma_k_
         _expect(gamma_k_shards[s], (wk,), bf, f"gamma_k_shards[{s}]")
         _expect(out_q_shards[s], (T, wq), bf, f"out_q_shards[{s}]")
         _expect(out_k_shards[s], (T, wk), bf, f"out_k_shards[{s}]")
-    _check(lib.qknorm_baseline_two_pass_static(_array(q_shards, S), _array(k_shards, S), _array(gamma_q_shards, S),
-                                               _array(gamma_k_shards, S), S, T, wq * S, wk * S, float(eps),
-                                               _array(out_q_shards, S), _array(out_k_shards, S), _stream(stream)))
+    _invoke(lib.qknorm_baseline_two_pass_static,
+            [_array(q_shards, S), _array(k_shards, S), _array(gamma_q_shards, S), _array(gamma_k_shards, S), S, T,
+             wq * S, wk * S, float(eps), _array(out_q_shards, S), _array(out_k_shards, S)], stream,
+            (q_shards, k_shards, gamma_q_shards, gamma_k_shards, out_q_shards, out_k_shards))
     return out_q_shards, out_k_shards
 
 

@@ -221,3 +221,25 @@ def test_no_bounded_wait_ever_ran_out(libqknorm):
     w = next(x for x in SMALL if x.name == "s_prefill_gqa")
     run_case(w, 8)
     assert binding.device_error_word() == 0
+
+
+def test_prepared_call_repeats_the_same_c_call(libqknorm):
+    """binding.prepared marshals once; the object makes the identical call again and again."""
+    w = next(x for x in SMALL if x.name == "s_prefill_gqa")
+    inp = W.make_inputs(w)
+    S = 8
+    qs = [t.cuda() for t in W.shard_columns(inp["q"], S)]
+    ks = [t.cuda() for t in W.shard_columns(inp["k"], S)]
+    gq = [t.cuda() for t in W.shard_columns(inp["gamma_q"], S)]
+    gk = [t.cuda() for t in W.shard_columns(inp["gamma_k"], S)]
+    n0 = binding.launch_count()
+    call = binding.prepared(binding.qknorm_fwd_sharded, qs, ks, gq, gk, w.eps)
+    assert binding.launch_count() == n0                 # preparing launches nothing
+    oq, ok = call.outputs
+    call()
+    call()
+    torch.cuda.synchronize()
+    assert binding.launch_count() == n0 + 2
+    ref = H.oracle_unsharded(inp, w.eps)
+    H.compare_output(H.bits(W.unshard_columns([t.cpu() for t in oq])), ref["q"]["y"], "prepared q")
+    H.compare_output(H.bits(W.unshard_columns([t.cpu() for t in ok])), ref["k"]["y"], "prepared k")

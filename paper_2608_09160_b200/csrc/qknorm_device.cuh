@@ -77,6 +77,7 @@ __device__ __forceinline__ uint32_t e4m3_pack2(float lo, float hi) {
 struct IoBf16 {
   static constexpr int kBytes = 2;       // bytes per element
   static constexpr int kGammaVecs = 1;   // 16-byte bf16 gamma vectors per 16-byte activation chunk
+  static constexpr bool kF16Gamma = false;  // no fp16 copy of gamma: bf16 * bf16 has its own mixed FMA
   // adds the squares of the word's elements to two accumulators
   static __device__ __forceinline__ void sumsq_word(uint32_t w, float& a, float& b) { fma_bf16x2_sq(w, a, b); }
   // (x * gamma) * r for one 16-byte chunk; g1 is unused
@@ -92,6 +93,9 @@ struct IoBf16 {
     o.w = bf_pack(p.x, p.y);
     return o;
   }
+  static __device__ __forceinline__ uint4 scale_chunk_g16(const uint4& x, const uint4& g0, const uint4& g1, float2 r2) {
+    return scale_chunk(x, g0, g1, r2);  // never selected (kF16Gamma is false)
+  }
   static __device__ __forceinline__ float load(const void* base, long long i) {
     return __uint_as_float(((uint32_t) reinterpret_cast<const uint16_t*>(base)[i]) << 16);
   }
@@ -101,9 +105,55 @@ struct IoBf16 {
   }
 };
 
+// (x_lo * g_lo, x_hi * g_hi) in fp32 for fp16 pairs; exact when x came from E4M3 (4 significant
+// bits) and g from bf16 (8 significant bits).  The addend is -0 so that a product of -0 keeps its sign.
+__device__ __forceinline__ float2 mul_f16x2(uint32_t x, uint32_t g) {
+  float2 p;
+  asm("{\n\t.reg .b16 xl, xh, gl, gh;\n\t"
+      "mov.b32 {xl, xh}, %2;\n\t"
+      "mov.b32 {gl, gh}, %3;\n\t"
+      "fma.rn.f32.f16 %0, xl, gl, 0f80000000;\n\t"
+      "fma.rn.f32.f16 %1, xh, gh, 0f80000000;\n\t}"
+      : "=f"(p.x), "=f"(p.y)
+      : "r"(x), "r"(g));
+  return p;
+}
+
+// Is this bf16 value exactly an fp16 value?  Zero, or a normal bf16 with exponent in [-17, 15]
+// (below -14 it lands on fp16 subnormals, whose spacing 2^-24 still holds 8 significant bits down
+// to 2^-17).  Infinities, NaNs and anything else answer no.
+__device__ __forceinline__ bool bf16_fits_f16(uint32_t b16) {
+  const uint32_t e = (b16 >> 7) & 0xffu, m = b16 & 0x7fu;
+  return (e == 0u && m == 0u) || (e >= 127u - 17u && e <= 127u + 15u);
+}
+__device__ __forceinline__ bool bf16x2_fits_f16(uint32_t w) { return bf16_fits_f16(w & 0xffffu) && bf16_fits_f16(w >> 16); }
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) {  // exact when bf16x2_fits_f16(w)
+  const __half2 h = __floats2half2_rn(bf_lo(w), bf_hi(w));
+  return *reinterpret_cast<const uint32_t*>(&h);
+}
+
 struct IoE4m3 {
   static constexpr int kBytes = 1;
   static constexpr int kGammaVecs = 2;   // 16 elements per chunk need 32 bytes of bf16 gamma
+  // When every gamma value is also an fp16 value (any realistic norm weight), the kernel keeps an
+  // fp16 copy of gamma and forms x * gamma with the fp16 mixed FMA: the product is exact either
+  // way, so the result is bit-identical to the bf16-gamma path, at fewer instructions.
+  static constexpr bool kF16Gamma = true;
+  static __device__ __forceinline__ uint32_t scale_word_g16(uint32_t x, uint32_t g01, uint32_t g23, float2 r2) {
+    uint32_t f01, f23;
+    e4m3x4_to_f16x2(x, f01, f23);
+    const float2 o01 = __fmul2_rn(mul_f16x2(f01, g01), r2);
+    const float2 o23 = __fmul2_rn(mul_f16x2(f23, g23), r2);
+    return e4m3_pack2(o01.x, o01.y) | (e4m3_pack2(o23.x, o23.y) << 16);
+  }
+  static __device__ __forceinline__ uint4 scale_chunk_g16(const uint4& x, const uint4& g0, const uint4& g1, float2 r2) {
+    uint4 o;
+    o.x = scale_word_g16(x.x, g0.x, g0.y, r2);
+    o.y = scale_word_g16(x.y, g0.z, g0.w, r2);
+    o.z = scale_word_g16(x.z, g1.x, g1.y, r2);
+    o.w = scale_word_g16(x.w, g1.z, g1.w, r2);
+    return o;
+  }
   static __device__ __forceinline__ void sumsq_word(uint32_t w, float& a, float& b) {
     uint32_t f01, f23;
     e4m3x4_to_f16x2(w, f01, f23);

@@ -41,6 +41,8 @@
 // Every mbarrier wait is bounded (about one second); a wait that runs out records
 // an error word and the warp leaves.
 #pragma once
+#include <type_traits>
+
 #include "qknorm_ring.cuh"
 #include "qknorm_rowmap.cuh"
 
@@ -129,10 +131,12 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
 
   // gamma, once per CTA (the first rows are already on their way): slot j of lane `lane`
   // holds the GV bf16 vectors that go with the lane's j-th chunk; slots dealt round-robin to the warps
+  bool gamma_f16 = false;
   {
     const uint4* gq = reinterpret_cast<const uint4*>(P.q.gamma[ss]) + (size_t)l * GV;
     const uint4* gk = reinterpret_cast<const uint4*>(P.k.gamma[ss]) + (size_t)l * GV;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    bool fits = true;
     for (int j = warp; j < L; j += cta_warps) {
 #pragma unroll
       for (int v = 0; v < GV; ++v) {
@@ -140,10 +144,30 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
         if (j < nvq) gv = __ldg(gq + (size_t)j * g * GV + v);
         else if (j >= wa.nq4 && j - wa.nq4 < nvk) gv = __ldg(gk + (size_t)(j - wa.nq4) * g * GV + v);
         gsm[j * GV + v][lane] = gv;
+        if (IO::kF16Gamma)
+          fits = fits && bf16x2_fits_f16(gv.x) && bf16x2_fits_f16(gv.y) && bf16x2_fits_f16(gv.z) && bf16x2_fits_f16(gv.w);
+      }
+    }
+    if (IO::kF16Gamma) {
+      // every gamma value of the CTA is also an fp16 value: keep gamma as fp16 (each thread
+      // converts the entries it wrote) and multiply with the fp16 mixed FMA
+      gamma_f16 = __syncthreads_and(fits ? 1 : 0) != 0;
+      if (gamma_f16) {
+        for (int j = warp; j < L; j += cta_warps) {
+#pragma unroll
+          for (int v = 0; v < GV; ++v) {
+            uint4 gv = gsm[j * GV + v][lane];
+            gv.x = bf16x2_to_f16x2(gv.x);
+            gv.y = bf16x2_to_f16x2(gv.y);
+            gv.z = bf16x2_to_f16x2(gv.z);
+            gv.w = bf16x2_to_f16x2(gv.w);
+            gsm[j * GV + v][lane] = gv;
+          }
+        }
       }
     }
   }
-  __syncthreads();  // the only block-level barrier
+  __syncthreads();  // the last block-level barrier
 
 
   // ---- loop-invariant per-lane offsets ------------------------------------------------------------
@@ -237,20 +261,27 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
     // ---- Phases B/C: (x * gamma) * RMS^-1, the one write ------------------------------------------------
     unsigned char* dq_ = yq + (unsigned long long)t * q_row;
     unsigned char* dk_ = yk + (unsigned long long)t * k_row;
+    auto store_pass = [&](auto f16_gamma) {  // the branch on the gamma format stays outside the slot loops
 #pragma unroll
-    for (int jb = 0; jb < L; jb += 4) {
-      if (jb >= n_slots) break;
-      const bool kpart = jb >= wa.nq4;
-      const float r = kpart ? rk : rq;
-      const float2 r2 = make_float2(r, r);
-      unsigned char* dst = kpart ? dk_ + (size_t)(jb - wa.nq4) * sstride : dq_ + (size_t)jb * sstride;
-      const int nv = kpart ? (EXACT ? wa.nk : nvk) - (jb - wa.nq4) : (EXACT ? wa.nq : nvq) - jb;
+      for (int jb = 0; jb < L; jb += 4) {
+        if (jb >= n_slots) break;
+        const bool kpart = jb >= wa.nq4;
+        const float r = kpart ? rk : rq;
+        const float2 r2 = make_float2(r, r);
+        unsigned char* dst = kpart ? dk_ + (size_t)(jb - wa.nq4) * sstride : dq_ + (size_t)jb * sstride;
+        const int nv = kpart ? (EXACT ? wa.nk : nvk) - (jb - wa.nq4) : (EXACT ? wa.nq : nvq) - jb;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint4 o = IO::scale_chunk(v[jb + i], gsm[(jb + i) * GV][lane], gsm[(jb + i) * GV + GV - 1][lane], r2);
-        if (i < nv) st_stream(reinterpret_cast<uint4*>(dst + (size_t)i * sstride), o);
+        for (int i = 0; i < 4; ++i) {
+          const uint4 ga = gsm[(jb + i) * GV][lane], gb = gsm[(jb + i) * GV + GV - 1][lane];
+          uint4 o;
+          if constexpr (decltype(f16_gamma)::value) o = IO::scale_chunk_g16(v[jb + i], ga, gb, r2);
+          else o = IO::scale_chunk(v[jb + i], ga, gb, r2);
+          if (i < nv) st_stream(reinterpret_cast<uint4*>(dst + (size_t)i * sstride), o);
+        }
       }
-    }
+    };
+    if (IO::kF16Gamma && gamma_f16) store_pass(std::true_type{});
+    else store_pass(std::false_type{});
   }
 }
 

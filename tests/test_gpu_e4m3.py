@@ -126,3 +126,22 @@ def test_full_size_e4m3(libqknorm, name):
         got = np.concatenate([W.e4m3_bits(t.cpu()[idx].contiguous()) for t in outs], axis=1)
         rate = compare_e4m3(got, np.concatenate(ref["y"], axis=1), f"{name}/e4m3/{nm}")
         print(f"{name} e4m3 {nm}: rate at distance 1 {rate:.2e}")
+
+
+def test_e4m3_gamma_outside_fp16_takes_the_bf16_gamma_path(libqknorm):
+    """The prefill kernel keeps an fp16 copy of gamma when every value fits fp16; one value that
+    does not (2^-20, 1e5) must switch the whole call to the bf16-gamma arithmetic with the same result."""
+    w = W.Workload("e_wide_gamma", tokens=700, dq=2048, dk=512, shards=(1,), seed=31, sigma=1.5)
+    inp = W.make_inputs_e4m3(w)
+    gq = inp["gamma_q"].clone()
+    gq[5] = 2.0 ** -20
+    gq[77] = 1.0e5
+    gq[300] = -(2.0 ** -18)
+    ref_q = oracle.rmsnorm_e4m3([W.e4m3_bits(inp["q"])], [W.bf16_bits(gq)], w.eps)["y"][0]
+    ref_k = oracle.rmsnorm_e4m3([W.e4m3_bits(inp["k"])], [W.bf16_bits(inp["gamma_k"])], w.eps)["y"][0]
+    oq, ok = binding.qknorm_fwd_e4m3(inp["q"].cuda(), inp["k"].cuda(), gq.cuda(), inp["gamma_k"].cuda(), w.eps)
+    torch.cuda.synchronize()
+    assert binding.last_variant() == "warp"
+    compare_e4m3(W.e4m3_bits(oq.cpu()), ref_q, "wide gamma q")
+    compare_e4m3(W.e4m3_bits(ok.cpu()), ref_k, "wide gamma k")
+    assert (W.e4m3_bits(oq.cpu())[:, 77] & 0x7F == 0x7E).mean() > 0.5     # 1e5 * x saturates

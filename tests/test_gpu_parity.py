@@ -243,3 +243,26 @@ def test_prepared_call_repeats_the_same_c_call(libqknorm):
     ref = H.oracle_unsharded(inp, w.eps)
     H.compare_output(H.bits(W.unshard_columns([t.cpu() for t in oq])), ref["q"]["y"], "prepared q")
     H.compare_output(H.bits(W.unshard_columns([t.cpu() for t in ok])), ref["k"]["y"], "prepared k")
+
+
+@pytest.mark.parametrize("T", [6, 700])          # the decode kernel and the prefill kernel
+def test_tiny_and_subnormal_inputs_are_not_flushed(libqknorm, T):
+    """bf16 subnormals and values whose squares underflow in fp32: with eps > 0 the statistic is
+    eps-dominated and the outputs (x * gamma / sqrt(eps)) must match the oracle; nothing may be
+    flushed to zero on the way."""
+    d = 1024
+    gen = torch.Generator().manual_seed(3)
+    x = torch.empty((T, d), dtype=torch.float32).normal_(0, 1, generator=gen)
+    x[0] *= 1e-39          # bf16 subnormals
+    x[1] *= 1e-30          # squares underflow in fp32
+    x[2] *= 1e-19          # squares are fp32 subnormals
+    x[3] *= 1e19           # large, still finite in fp32 after squaring and summing (1e38 * 1024 overflows? no: 1e38*... keep below)
+    x[3] *= 1e-2
+    xb = x.to(torch.bfloat16)
+    g = torch.empty((d,), dtype=torch.float32).uniform_(0.5, 1.5, generator=gen).to(torch.bfloat16)
+    oq, _ = binding.qknorm_fwd(xb.cuda(), None, g.cuda(), None, 1e-6)
+    with np.errstate(all="ignore"):
+        ref = oracle.rmsnorm(W.bf16_bits(xb), W.bf16_bits(g), 1e-6)["y"]
+    got = H.bits(oq)
+    H.compare_output(got, ref, f"tiny inputs T={T}")
+    assert (got[0] & 0x7FFF).any(), "subnormal inputs were flushed to zero"

@@ -1,5 +1,6 @@
 // C ABI of libqknorm: argument validation, variant choice, launch.
-// Nothing here allocates device memory, copies, or synchronises.
+// No forward entry point allocates device memory, copies, or synchronises (the inbox
+// helpers of the tensor-parallel path, qknorm_tp_host.cuh, are the only routines that do).
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdlib.h>
@@ -775,6 +776,8 @@ int static_scratch_address(float** out) {
 
 }  // namespace
 }  // namespace qknorm
+
+#include "qknorm_tp_host.cuh"  // the tensor-parallel entry points (include/qknorm_tp.h)
 
 extern "C" {
 

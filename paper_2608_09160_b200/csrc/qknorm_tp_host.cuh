@@ -1,0 +1,277 @@
+// Host side of the tensor-parallel entry points (include/qknorm_tp.h): validation,
+// grid choice and the cooperative launch of tp_kernel, plus the inbox helpers.
+// Included by qknorm_api.cu after its own helpers (device cache, occupancy cache,
+// overlap test), which it uses.
+#pragma once
+#include "../../include/qknorm_tp.h"
+#include "qknorm_tp.cuh"
+
+namespace qknorm {
+
+#define QKNORM_DECL_TP_L(l)     \
+  TpKernel tp_kernel_bf16_l##l(); \
+  TpKernel tp_kernel_e4m3_l##l();
+QKNORM_DECL_TP_L(4) QKNORM_DECL_TP_L(8) QKNORM_DECL_TP_L(12) QKNORM_DECL_TP_L(16) QKNORM_DECL_TP_L(20)
+QKNORM_DECL_TP_L(24) QKNORM_DECL_TP_L(28) QKNORM_DECL_TP_L(32) QKNORM_DECL_TP_L(36) QKNORM_DECL_TP_L(40)
+
+TpKernel tp_kernel_for(int l, int elem_bytes) {
+#define QKNORM_CASE_TP_L(l) \
+  case l: return elem_bytes == 1 ? tp_kernel_e4m3_l##l() : tp_kernel_bf16_l##l();
+  switch (l) {
+    QKNORM_CASE_TP_L(4) QKNORM_CASE_TP_L(8) QKNORM_CASE_TP_L(12) QKNORM_CASE_TP_L(16) QKNORM_CASE_TP_L(20)
+    QKNORM_CASE_TP_L(24) QKNORM_CASE_TP_L(28) QKNORM_CASE_TP_L(32) QKNORM_CASE_TP_L(36) QKNORM_CASE_TP_L(40)
+    default: return nullptr;
+  }
+#undef QKNORM_CASE_TP_L
+}
+
+namespace {
+
+int tp_inbox_bytes(int num_ranks, long long cap, long long* bytes) {
+  if (!bytes) return QKNORM_ERR_NULL;
+  if (num_ranks < 1 || num_ranks > kMaxShards) return QKNORM_ERR_SHARDS;
+  if (cap < 1 || cap > (1LL << 31)) return QKNORM_ERR_SHAPE;
+  *bytes = 8LL * (kTpHeaderWords + 4LL * num_ranks * cap);
+  return QKNORM_OK;
+}
+
+int run_tp(int elem_bytes, const qknorm_tp_rank* ranks, int n_local, int N, long long T, long long cap,
+           int wq, int wk, const int64_t* ld, float eps, uint32_t epoch, uint32_t wait_limit_us,
+           cudaStream_t stream) {
+  if (N < 1 || N > kMaxShards || n_local < 1 || n_local > N) return QKNORM_ERR_SHARDS;
+  if (T < 0 || wq < 0 || wk < 0 || cap < 1 || T > cap || cap > (1LL << 31)) return QKNORM_ERR_SHAPE;
+  if ((long long)wq * N > kMaxDim || (long long)wk * N > kMaxDim) return QKNORM_ERR_SHAPE;
+  if (!(eps >= 0.0f)) return QKNORM_ERR_EPS;
+  if (T == 0) return QKNORM_OK;
+  if (wq == 0 && wk == 0) return QKNORM_ERR_SHAPE;
+  if (epoch == 0u) return QKNORM_ERR_SHAPE;
+  if (!ranks) return QKNORM_ERR_NULL;
+
+  TpParams P;
+  memset(&P, 0, sizeof(P));
+  P.n_local = n_local;
+  P.N = N;
+  P.T = T;
+  P.cap = cap;
+  P.wq = wq;
+  P.wk = wk;
+  P.ldxq = (ld && ld[0]) ? ld[0] : wq;
+  P.ldxk = (ld && ld[1]) ? ld[1] : wk;
+  P.ldyq = (ld && ld[2]) ? ld[2] : wq;
+  P.ldyk = (ld && ld[3]) ? ld[3] : wk;
+  if (P.ldxq < wq || P.ldyq < wq || P.ldxk < wk || P.ldyk < wk) return QKNORM_ERR_SHAPE;
+  P.inv_dq = wq ? 1.0f / (float)(wq * N) : 0.0f;
+  P.inv_dk = wk ? 1.0f / (float)(wk * N) : 0.0f;
+  P.eps = eps;
+  P.epoch = epoch;
+  P.wait_ns = 1000ull * (wait_limit_us ? wait_limit_us : 1000000u);
+
+  const uintptr_t eb = (uintptr_t)elem_bytes;
+  if ((wq * elem_bytes) % 16 || (wk * elem_bytes) % 16) return QKNORM_ERR_ALIGN;
+  if ((P.ldxq * elem_bytes) % 16 || (P.ldxk * elem_bytes) % 16 || (P.ldyq * elem_bytes) % 16 || (P.ldyk * elem_bytes) % 16)
+    return QKNORM_ERR_ALIGN;
+  long long inbox_bytes = 0;
+  int rc = tp_inbox_bytes(N, cap, &inbox_bytes);
+  if (rc != QKNORM_OK) return rc;
+
+  unsigned seen = 0;
+  Region outs[2 * kMaxShards], ins[2 * kMaxShards], others[8 * kMaxShards];
+  int n_out = 0, n_other = 0;
+  for (int i = 0; i < n_local; ++i) {
+    const qknorm_tp_rank& a = ranks[i];
+    TpRank& r = P.r[i];
+    if (a.rank < 0 || a.rank >= N || (seen >> a.rank) & 1u) return QKNORM_ERR_SHARDS;
+    seen |= 1u << a.rank;
+    if (wq && (!a.q || !a.gamma_q || !a.out_q)) return QKNORM_ERR_NULL;
+    if (wk && (!a.k || !a.gamma_k || !a.out_k)) return QKNORM_ERR_NULL;
+    if (!a.inbox || (N > 1 && !a.peer_inbox)) return QKNORM_ERR_NULL;
+    r.rank = a.rank;
+    r.xq = wq ? a.q : nullptr;
+    r.xk = wk ? a.k : nullptr;
+    r.gq = wq ? (const uint16_t*)a.gamma_q : nullptr;
+    r.gk = wk ? (const uint16_t*)a.gamma_k : nullptr;
+    r.yq = wq ? a.out_q : nullptr;
+    r.yk = wk ? a.out_k : nullptr;
+    r.rstd_q = wq ? a.rstd_q : nullptr;
+    r.rstd_k = wk ? a.rstd_k : nullptr;
+    r.partial_q = wq ? a.partial_q : nullptr;
+    r.partial_k = wk ? a.partial_k : nullptr;
+    r.inbox = (unsigned long long*)a.inbox;
+    if (!aligned16(r.xq) || !aligned16(r.xk) || !aligned16(r.gq) || !aligned16(r.gk) || !aligned16(r.yq) || !aligned16(r.yk))
+      return QKNORM_ERR_ALIGN;
+    if (((uintptr_t)a.inbox) & 7u) return QKNORM_ERR_ALIGN;
+    if ((((uintptr_t)a.rstd_q) | ((uintptr_t)a.rstd_k) | ((uintptr_t)a.partial_q) | ((uintptr_t)a.partial_k)) & 3u)
+      return QKNORM_ERR_ALIGN;
+    for (int p = 0; p < N; ++p) {
+      if (p == a.rank) continue;
+      const void* peer = a.peer_inbox[p];
+      if (!peer) return QKNORM_ERR_NULL;
+      if (((uintptr_t)peer) & 7u) return QKNORM_ERR_ALIGN;
+      r.peer_inbox[p] = (unsigned long long*)peer;
+    }
+    const uintptr_t rows = (uintptr_t)T;
+    if (wq) {
+      ins[n_out] = {(uintptr_t)a.q, rows, (uintptr_t)wq * eb, (uintptr_t)P.ldxq * eb};
+      outs[n_out++] = {(uintptr_t)a.out_q, rows, (uintptr_t)wq * eb, (uintptr_t)P.ldyq * eb};
+      others[n_other++] = {(uintptr_t)a.gamma_q, 1, (uintptr_t)wq * 2u, (uintptr_t)wq * 2u};
+    }
+    if (wk) {
+      ins[n_out] = {(uintptr_t)a.k, rows, (uintptr_t)wk * eb, (uintptr_t)P.ldxk * eb};
+      outs[n_out++] = {(uintptr_t)a.out_k, rows, (uintptr_t)wk * eb, (uintptr_t)P.ldyk * eb};
+      others[n_other++] = {(uintptr_t)a.gamma_k, 1, (uintptr_t)wk * 2u, (uintptr_t)wk * 2u};
+    }
+    others[n_other++] = {(uintptr_t)a.inbox, 1, (uintptr_t)inbox_bytes, (uintptr_t)inbox_bytes};
+    float* aux[4] = {r.rstd_q, r.rstd_k, r.partial_q, r.partial_k};
+    for (float* x : aux)
+      if (x) others[n_other++] = {(uintptr_t)x, 1, 4u * rows, 4u * rows};
+  }
+  // an output may be exactly its own input; any other overlap with a buffer of the call is an error
+  for (int i = 0; i < n_out; ++i) {
+    for (int j = 0; j < n_out; ++j) {
+      if (may_overlap(outs[i], ins[j]) && !(i == j && same_region(outs[i], ins[j]))) return QKNORM_ERR_ALIAS;
+      if (j != i && may_overlap(outs[i], outs[j])) return QKNORM_ERR_ALIAS;
+    }
+    for (int j = 0; j < n_other; ++j)
+      if (may_overlap(outs[i], others[j])) return QKNORM_ERR_ALIAS;
+  }
+
+  // chunk slots per lane: the whole warp serves the rank's one slice of each tensor
+  const int cq = wq * elem_bytes / 16, ck = wk * elem_bytes / 16;
+  P.nq = (cq + 31) / 32;
+  P.nk = (ck + 31) / 32;
+  P.nq4 = round_up(P.nq, 4);
+  const int l = warp_round_up_l(P.nq4 + P.nk);
+  TpKernel fn = l > 0 ? tp_kernel_for(l, elem_bytes) : nullptr;
+  if (!fn) return QKNORM_ERR_SHAPE;  // slice rows too long for one warp
+  P.k_base = wq * elem_bytes;
+  P.zero_off = P.k_base + wk * elem_bytes;
+  P.stage_bytes = round_up(P.zero_off + 16, 128);
+
+  const DeviceInfo* dev = nullptr;
+  rc = current_device(&dev);
+  if (rc != QKNORM_OK) return rc;
+  const int warps = kWarpMaxCtaWarps;
+  const int smem = warps * P.stage_bytes;
+  rc = allow_dynamic_smem((const void*)fn, smem);
+  if (rc != QKNORM_OK) return rc;
+  int resident = 1;
+  rc = resident_blocks((const void*)fn, warps * 32, smem, &resident);
+  if (rc != QKNORM_OK) return rc;
+  const int cap_ctas = env_int("QKNORM_TP_CTAS_PER_SM", 0);
+  if (cap_ctas > 0 && cap_ctas < resident) resident = cap_ctas;
+  // bounded grid (Section III-D): every CTA of every rank served here is resident at once
+  long long per_rank = (long long)resident * dev->sm_count / n_local;
+  const long long needed = (T + warps - 1) / warps;
+  if (per_rank > needed) per_rank = needed;
+  if (per_rank < 1) return QKNORM_ERR_SHARDS;  // more local ranks than resident CTAs
+  const unsigned grid = (unsigned)(per_rank * n_local);
+  void* args[] = {(void*)&P};
+  cudaError_t e = cudaLaunchCooperativeKernel((const void*)fn, dim3(grid), dim3(warps * 32), args, (size_t)smem, stream);
+  if (e != cudaSuccess) return set_cuda_error(e);
+  return finish_launch("tp");
+}
+
+}  // namespace
+}  // namespace qknorm
+
+extern "C" {
+
+int qknorm_tp_inbox_bytes(int32_t num_ranks, int64_t token_capacity, int64_t* bytes) {
+  long long b = 0;
+  const int rc = qknorm::tp_inbox_bytes(num_ranks, token_capacity, bytes ? &b : nullptr);
+  if (rc == QKNORM_OK) *bytes = b;
+  return rc;
+}
+
+int qknorm_fwd_tp(const qknorm_tp_rank* ranks, int32_t n_local, int32_t num_ranks, int64_t tokens,
+                  int64_t token_capacity, int32_t wq, int32_t wk, const int64_t* ld, float eps, uint32_t epoch,
+                  uint32_t wait_limit_us, void* stream) {
+  return qknorm::run_tp(2, ranks, n_local, num_ranks, tokens, token_capacity, wq, wk, ld, eps, epoch,
+                        wait_limit_us, (cudaStream_t)stream);
+}
+
+int qknorm_fwd_tp_e4m3(const qknorm_tp_rank* ranks, int32_t n_local, int32_t num_ranks, int64_t tokens,
+                       int64_t token_capacity, int32_t wq, int32_t wk, const int64_t* ld, float eps, uint32_t epoch,
+                       uint32_t wait_limit_us, void* stream) {
+  return qknorm::run_tp(1, ranks, n_local, num_ranks, tokens, token_capacity, wq, wk, ld, eps, epoch,
+                        wait_limit_us, (cudaStream_t)stream);
+}
+
+int qknorm_tp_status(const void* inbox, int32_t* out) {
+  if (!inbox || !out) return QKNORM_ERR_NULL;
+  cudaError_t e = cudaMemcpy(out, inbox, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  return QKNORM_OK;
+}
+
+int qknorm_tp_clear_status(void* inbox, void* stream) {
+  if (!inbox) return QKNORM_ERR_NULL;
+  cudaError_t e = cudaMemsetAsync(inbox, 0, 8 * qknorm::kTpHeaderWords, (cudaStream_t)stream);
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  return QKNORM_OK;
+}
+
+int qknorm_tp_inbox_create(int32_t num_ranks, int64_t token_capacity, void** out) {
+  if (!out) return QKNORM_ERR_NULL;
+  long long bytes = 0;
+  const int rc = qknorm::tp_inbox_bytes(num_ranks, token_capacity, &bytes);
+  if (rc != QKNORM_OK) return rc;
+  void* p = nullptr;
+  cudaError_t e = cudaMalloc(&p, (size_t)bytes);
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  e = cudaMemset(p, 0, (size_t)bytes);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    cudaFree(p);
+    return qknorm::set_cuda_error(e);
+  }
+  *out = p;
+  return QKNORM_OK;
+}
+
+int qknorm_tp_inbox_zero(void* inbox, int32_t num_ranks, int64_t token_capacity, void* stream) {
+  if (!inbox) return QKNORM_ERR_NULL;
+  long long bytes = 0;
+  const int rc = qknorm::tp_inbox_bytes(num_ranks, token_capacity, &bytes);
+  if (rc != QKNORM_OK) return rc;
+  cudaError_t e = cudaMemsetAsync(inbox, 0, (size_t)bytes, (cudaStream_t)stream);
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  return QKNORM_OK;
+}
+
+int qknorm_tp_inbox_destroy(void* inbox) {
+  if (!inbox) return QKNORM_OK;
+  cudaError_t e = cudaFree(inbox);
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  return QKNORM_OK;
+}
+
+int qknorm_tp_ipc_export(const void* inbox, unsigned char* handle) {
+  static_assert(sizeof(cudaIpcMemHandle_t) == QKNORM_TP_IPC_HANDLE_BYTES, "handle size");
+  if (!inbox || !handle) return QKNORM_ERR_NULL;
+  cudaIpcMemHandle_t h;
+  cudaError_t e = cudaIpcGetMemHandle(&h, const_cast<void*>(inbox));
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  memcpy(handle, &h, sizeof(h));
+  return QKNORM_OK;
+}
+
+int qknorm_tp_ipc_open(const unsigned char* handle, void** out) {
+  if (!handle || !out) return QKNORM_ERR_NULL;
+  cudaIpcMemHandle_t h;
+  memcpy(&h, handle, sizeof(h));
+  void* p = nullptr;
+  cudaError_t e = cudaIpcOpenMemHandle(&p, h, cudaIpcMemLazyEnablePeerAccess);
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  *out = p;
+  return QKNORM_OK;
+}
+
+int qknorm_tp_ipc_close(void* mapped) {
+  if (!mapped) return QKNORM_OK;
+  cudaError_t e = cudaIpcCloseMemHandle(mapped);
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  return QKNORM_OK;
+}
+
+}  // extern "C"

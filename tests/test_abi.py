@@ -10,16 +10,25 @@ from paper_2608_09160_b200 import binding
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 HEADER = os.path.join(ROOT, "include", "qknorm.h")
+HEADER_TP = os.path.join(ROOT, "include", "qknorm_tp.h")
 
 
-def declared_functions():
-    src = open(HEADER).read()
+def declared_functions(header=HEADER):
+    src = open(header).read()
     src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
     return sorted(set(re.findall(r"\b(qknorm_[a-z0-9_]+)\s*\(", src)))
 
 
 def test_header_and_binding_agree_on_exports():
     assert declared_functions() == sorted(binding.EXPORTS)
+
+
+def test_tensor_parallel_header_and_binding_agree_on_exports(libqknorm):
+    from paper_2608_09160_b200 import tp
+    names = [n for n in declared_functions(HEADER_TP) if n != "qknorm_tp_rank"]
+    assert names == sorted(tp.EXPORTS)
+    for name in names:
+        assert hasattr(libqknorm, name), name
 
 
 def test_library_exports_every_declared_symbol(libqknorm):

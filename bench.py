@@ -335,6 +335,36 @@ def config_table(steps: int, warmup: int, peak: float, skip: str):
             torch.cuda.empty_cache()
     rows.update(variant_rows(steps, warmup, peak))
     rows.update(baseline_rows(steps, warmup, peak))
+    rows.update(tp_rows(steps, warmup, peak))
+    return rows
+
+
+def tp_rows(steps: int, warmup: int, peak: float):
+    """The tensor-parallel kernel (Algorithm 1 with its scalar exchange) with all N ranks on this
+    one GPU: one cooperative launch serves every rank, scalars go through the ranks' inboxes in
+    device memory.  Same bytes as the logical-shard call, so the difference to it is what the
+    exchange protocol itself costs when the link is free."""
+    from paper_2608_09160_b200 import binding, tp
+    rows = {}
+    for name, N in (("C3", 4), ("C4", 8), ("C5", 8)):
+        w = W.WORKLOADS[name]
+        inp = W.make_inputs(w)
+        dev = {k: [t.cuda() for t in W.shard_columns(inp[k], N)] for k in ("q", "k", "gamma_q", "gamma_k")}
+        del inp
+        grp = tp.EmulatedGroup(N, token_capacity=w.tokens)
+        bufs = grp.buffers(dev["q"], dev["k"], dev["gamma_q"], dev["gamma_k"], out_q=dev["q"], out_k=dev["k"])
+        call = grp.prepare(bufs, w.eps)
+        ts = time_calls(lambda: call(grp.epochs.next()), max(steps, 10), max(warmup, 3))
+        med = statistics.median(ts)
+        gbs = w.algorithmic_bytes / (med * 1e-3) / 1e9
+        ok = all(tp.status(b)["status"] == tp.STATUS_OK for b in grp.inboxes)
+        rows[f"{name}/TP{N}-one-GPU-emulation/in-place"] = {
+            "us_median": round(med * 1e3, 3), "us_min": round(min(ts) * 1e3, 3), "GBps": round(gbs, 1),
+            "frac_measured_peak": round(gbs / peak, 4), "frac_nominal_8TBps": round(gbs / NOMINAL_HBM_GBS, 4),
+            "bytes": w.algorithmic_bytes, "variant": binding.last_variant(), "l2": "inputs larger than L2",
+            "exchange_bytes_per_call": 16 * w.tokens * N * (N - 1), "all_waits_completed": ok}
+        del dev, bufs, call, grp
+        torch.cuda.empty_cache()
     return rows
 
 

@@ -16,13 +16,13 @@
 //    double-buffered by epoch parity: a rank can run at most one call ahead of a peer
 //    (it needs the peer's scalars of call c+1 to finish c+1), so what it writes for c+2
 //    lands in the half the peer finished with c.
-//  * no warp is set aside for communication.  The kernel is the warp-per-token design of
-//    the single-GPU path: a warp has its NEXT row in flight (TMA bulk copy into its own
-//    shared-memory stage) while it waits for the scalars of the current one, and the
-//    other warps of the SM (up to 32 for slice rows of <= 4 KB) cover the link latency.
-//  * lanes 0..N-1 of the warp each talk to one peer: lane p stores to rank p's inbox and
-//    polls the slot rank p fills here, so the N-1 stores and N-1 polls of a token are
-//    one instruction each.
+//  * no warp is set aside for communication.  The kernel keeps the warp-level design of
+//    the single-GPU path: a warp has its NEXT tile of rows in flight (TMA bulk copies into
+//    its own shared-memory stage) while it waits for the scalars of the current one, and
+//    the other warps of the SM cover the link latency.
+//  * a warp works on several tokens side by side (see tp_kernel), and one lane per
+//    (token, peer) pair carries the exchange: all pushes of a tile are one store
+//    instruction, all polls one loop.
 //
 // The launch is cooperative, so the driver itself refuses a grid whose CTAs are not all
 // resident (the bounded grid of Section III-D).  Every warp works through its tokens in
@@ -46,6 +46,7 @@
 
 namespace qknorm {
 
+constexpr int kTpRounds = 4;        // exchange rounds of 32 (token, rank) pairs: tile * N <= 128
 constexpr int kTpHeaderWords = 32;  // 256-byte header in front of the slots (64-bit words)
 
 // status codes in word 0 of the inbox header
@@ -82,8 +83,12 @@ struct TpParams {
   float eps;
   uint32_t epoch;         // != 0
   unsigned long long wait_ns;
+  int log_g;              // log2 of the lanes that serve one token (32 >> log_g tokens per warp tile)
   int nq, nk, nq4;        // chunk slots per lane: Q part, K part, first K slot
-  int stage_bytes, k_base, zero_off;
+  int stage_bytes;        // one warp's stage: the tile's Q rows, its K rows, 16 zero bytes
+  int q_row_stride;       // bytes between consecutive tokens' Q rows inside a stage (row + bank skew)
+  int k_row_stride;
+  int k_base, zero_off;
 };
 
 namespace ptx {
@@ -145,6 +150,14 @@ __device__ __forceinline__ bool tp_poll2(const unsigned long long* sq, const uns
   return true;
 }
 
+// A warp works on a TILE of R = 32 >> log_g consecutive tokens at a time: lane group s
+// (g = 32 / R lanes) serves token t0 + s, lane l of the group owns chunks l, l+g, ... of
+// that token's Q slice row and K slice row.  Slice rows are short (a few KB), so one token
+// per warp would spend most of its instructions on per-token work (barrier wait, copy
+// issue, shuffles, push, poll); with R tokens side by side that work is done once per tile:
+// one log2(g)-step shuffle tree gives all R scalars, ONE store instruction pushes R x (N-1)
+// scalars (lane p*R + r: token r to rank p), one poll loop collects them, N broadcasts per
+// tensor form all R sums.  When R * N exceeds 32 the pairs take up to kTpRounds rounds.
 template <int L, class IO>
 __global__ void __launch_bounds__(kWarpMaxCtaWarps * 32, tp_min_blocks(L, IO::kBytes))
 tp_kernel(const __grid_constant__ TpParams P) {
@@ -161,9 +174,13 @@ tp_kernel(const __grid_constant__ TpParams P) {
   const long long ctas = gridDim.x / (unsigned)P.n_local;
   int* const status = reinterpret_cast<int*>(R.inbox);
 
+  const int g = 1 << P.log_g;
+  const int tile = 32 >> P.log_g;  // tokens per tile
+  const int s = lane >> P.log_g;   // which token of the tile this lane serves
+  const int l = lane & (g - 1);
   const int cq = (P.wq * IO::kBytes) >> 4, ck = (P.wk * IO::kBytes) >> 4;  // 16-byte chunks per slice row
-  const int nvq = lane < cq ? (cq - lane + 31) >> 5 : 0;
-  const int nvk = lane < ck ? (ck - lane + 31) >> 5 : 0;
+  const int nvq = l < cq ? (cq - l + g - 1) >> P.log_g : 0;
+  const int nvk = l < ck ? (ck - l + g - 1) >> P.log_g : 0;
   const int n_slots = P.nq4 + P.nk;
 
   unsigned char* stage = tp_smem + (size_t)warp * P.stage_bytes;
@@ -175,47 +192,54 @@ tp_kernel(const __grid_constant__ TpParams P) {
     ptx::fence_proxy_async();
     *reinterpret_cast<uint4*>(stage + P.zero_off) = make_uint4(0u, 0u, 0u, 0u);
   }
-  // lane 0 fetches the Q slice row, lane 1 the K slice row
+  // lane i < tile fetches the Q slice row of token i of the tile, lane tile + i its K slice row
+  const bool issue_q = lane < tile;
+  const int is = issue_q ? lane : lane - tile;
   uint32_t my_bytes = 0, my_dst = 0;
   unsigned long long my_pitch = 0;
   const unsigned char* my_src = nullptr;
-  if (lane == 0 && cq) {
-    my_bytes = (uint32_t)P.wq * IO::kBytes;
-    my_pitch = (unsigned long long)P.ldxq * IO::kBytes;
-    my_src = reinterpret_cast<const unsigned char*>(R.xq);
-  } else if (lane == 1 && ck) {
-    my_bytes = (uint32_t)P.wk * IO::kBytes;
-    my_pitch = (unsigned long long)P.ldxk * IO::kBytes;
-    my_src = reinterpret_cast<const unsigned char*>(R.xk);
-    my_dst = (uint32_t)P.k_base;
+  if (lane < 2 * tile) {
+    if (issue_q && cq) {
+      my_bytes = (uint32_t)P.wq * IO::kBytes;
+      my_pitch = (unsigned long long)P.ldxq * IO::kBytes;
+      my_src = reinterpret_cast<const unsigned char*>(R.xq);
+      my_dst = (uint32_t)is * (uint32_t)P.q_row_stride;
+    } else if (!issue_q && ck) {
+      my_bytes = (uint32_t)P.wk * IO::kBytes;
+      my_pitch = (unsigned long long)P.ldxk * IO::kBytes;
+      my_src = reinterpret_cast<const unsigned char*>(R.xk);
+      my_dst = (uint32_t)P.k_base + (uint32_t)is * (uint32_t)P.k_row_stride;
+    }
   }
   const uint32_t row_bytes = ((uint32_t)P.wq + (uint32_t)P.wk) * IO::kBytes;
   const uint64_t policy = ptx::policy_evict_first();
-  auto arm = [&](long long t) {  // whole warp
-    if (lane == 0) ptx::mbar_arrive_expect_tx(bar, row_bytes);
+  auto arm = [&](long long t0) {  // whole warp; t0 = first token of the tile
+    const long long left = P.T - t0;
+    const int n = left < tile ? (int)left : tile;
+    if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)n * row_bytes);
     __syncwarp();
-    if (my_bytes) ptx::bulk_load(stage_u32 + my_dst, my_src + (unsigned long long)t * my_pitch, my_bytes, bar, policy);
+    if (my_bytes && is < n) ptx::bulk_load(stage_u32 + my_dst, my_src + (unsigned long long)(t0 + is) * my_pitch, my_bytes, bar, policy);
   };
 
   const int cta_warps = blockDim.x >> 5;
-  const long long first = cta * cta_warps + warp;
-  const long long step = ctas * cta_warps;
+  const long long first = (cta * cta_warps + warp) * tile;
+  const long long step = ctas * cta_warps * tile;
   __syncwarp();
   if (first < P.T) arm(first);
 
-  // gamma of the slice, once per CTA, as [chunk slot][lane]
+  // gamma of the slice, once per CTA, as [chunk slot][lane] (the same values in every lane group)
   bool gamma_f16 = false;
   {
-    const uint4* gq = reinterpret_cast<const uint4*>(R.gq) + (size_t)lane * GV;
-    const uint4* gk = reinterpret_cast<const uint4*>(R.gk) + (size_t)lane * GV;
+    const uint4* gq = reinterpret_cast<const uint4*>(R.gq) + (size_t)l * GV;
+    const uint4* gk = reinterpret_cast<const uint4*>(R.gk) + (size_t)l * GV;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
     bool fits = true;
     for (int j = warp; j < L; j += cta_warps) {
 #pragma unroll
       for (int v = 0; v < GV; ++v) {
         uint4 gv = zero;
-        if (j < nvq) gv = __ldg(gq + (size_t)j * 32 * GV + v);
-        else if (j >= P.nq4 && j - P.nq4 < nvk) gv = __ldg(gk + (size_t)(j - P.nq4) * 32 * GV + v);
+        if (j < nvq) gv = __ldg(gq + (size_t)j * g * GV + v);
+        else if (j >= P.nq4 && j - P.nq4 < nvk) gv = __ldg(gk + (size_t)(j - P.nq4) * g * GV + v);
         gsm[j * GV + v][lane] = gv;
         if (IO::kF16Gamma)
           fits = fits && bf16x2_fits_f16(gv.x) && bf16x2_fits_f16(gv.y) && bf16x2_fits_f16(gv.z) && bf16x2_fits_f16(gv.w);
@@ -240,44 +264,36 @@ tp_kernel(const __grid_constant__ TpParams P) {
   }
   __syncthreads();  // the last block-level barrier
 
-  // ---- the exchange: lane p < N talks to rank p --------------------------------------------------------
+  // ---- the exchange: pair number (rd * 32 + lane) = p * tile + r carries token r of the tile to and
+  // from rank p; kTpRounds rounds of 32 pairs cover tile * N <= 128 pairs ---------------------------
   const int parity = (int)(P.epoch & 1u);
-  const bool remote = lane < P.N && lane != R.rank;
-  unsigned long long* push_q = nullptr;        // where this rank's scalar goes in rank `lane`'s inbox
-  unsigned long long* push_k = nullptr;
-  const unsigned long long* poll_q = nullptr;  // where rank `lane`'s scalar lands in this rank's inbox
-  const unsigned long long* poll_k = nullptr;
-  if (remote) {
-    unsigned long long* peer = R.peer_inbox[lane];
-    if (cq) {
-      push_q = peer + tp_slot_index(parity, 0, R.rank, P.N, P.cap);
-      poll_q = R.inbox + tp_slot_index(parity, 0, lane, P.N, P.cap);
-    }
-    if (ck) {
-      push_k = peer + tp_slot_index(parity, 1, R.rank, P.N, P.cap);
-      poll_k = R.inbox + tp_slot_index(parity, 1, lane, P.N, P.cap);
-    }
-  }
+  const int xr = lane & (tile - 1);         // token of the tile this lane exchanges (the same in every round)
+  const int xp0 = lane >> (5 - P.log_g);    // rank this lane talks to in round 0; round rd: xp0 + rd * g
+  const long long slot_q_out = tp_slot_index(parity, 0, R.rank, P.N, P.cap) + xr;  // in a peer's inbox
+  const long long slot_k_out = tp_slot_index(parity, 1, R.rank, P.N, P.cap) + xr;
+  const int rounds = (tile * P.N + 31) >> 5;
   const unsigned long long tag = (unsigned long long)P.epoch << 32;
 
-  const uint32_t sq0 = stage_u32 + (uint32_t)lane * 16u;
-  const uint32_t sk0 = stage_u32 + (uint32_t)P.k_base + (uint32_t)lane * 16u;
+  const uint32_t sq0 = stage_u32 + (uint32_t)s * (uint32_t)P.q_row_stride + (uint32_t)l * 16u;
+  const uint32_t sk0 = stage_u32 + (uint32_t)P.k_base + (uint32_t)s * (uint32_t)P.k_row_stride + (uint32_t)l * 16u;
   const uint32_t szero = stage_u32 + (uint32_t)P.zero_off;
-  constexpr uint32_t sstride = 32u * 16u;
-  unsigned char* yq = reinterpret_cast<unsigned char*>(R.yq) + (size_t)lane * 16u;
-  unsigned char* yk = reinterpret_cast<unsigned char*>(R.yk) + (size_t)lane * 16u;
+  const uint32_t sstride = (uint32_t)g * 16u;
+  unsigned char* yq = reinterpret_cast<unsigned char*>(R.yq) + (size_t)l * 16u;
+  unsigned char* yk = reinterpret_cast<unsigned char*>(R.yk) + (size_t)l * 16u;
   const unsigned long long q_row = (unsigned long long)P.ldyq * IO::kBytes, k_row = (unsigned long long)P.ldyk * IO::kBytes;
 
   uint32_t phase = 0;
-  for (long long t = first; t < P.T; t += step) {
+  for (long long t0 = first; t0 < P.T; t0 += step) {
     if (!ptx::mbar_wait_bounded(bar, phase)) {
       if (lane == 0 && atomicCAS(status, kTpOk, kTpStageTimeout) == kTpOk) {
-        status[1] = (int)(t & 0x7fffffff);
+        status[1] = (int)(t0 & 0x7fffffff);
         status[2] = -1;
       }
       return;
     }
     phase ^= 1u;
+    const long long t = t0 + s;       // this lane group's token
+    const bool live = t < P.T;        // the last tile may be short: its stage rows are stale, never published
     // ---- drain the stage into registers --------------------------------------------------------
     uint4 v[L];
 #pragma unroll
@@ -289,7 +305,7 @@ tp_kernel(const __grid_constant__ TpParams P) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) v[jb + i] = ptx::lds128(i < nv ? base + (uint32_t)i * sstride : szero);
     }
-    // ---- Phase A: S_local of the Q slice and of the K slice -------------------------------------------
+    // ---- Phase A: S_local of the Q slice and of the K slice, one token per lane group --------------
     float2 aq = make_float2(0.f, 0.f), ak = make_float2(0.f, 0.f);
 #pragma unroll
     for (int jb = 0; jb < L; jb += 4) {
@@ -317,43 +333,76 @@ tp_kernel(const __grid_constant__ TpParams P) {
       else aq = __fadd2_rn(aq, b);
     }
     float pq = aq.x + aq.y, pk = ak.x + ak.y;
+    // the same tree in every lane of a group: all g lanes end with the same bits
+    if (g > 16) { pq += __shfl_xor_sync(0xffffffffu, pq, 16); pk += __shfl_xor_sync(0xffffffffu, pk, 16); }
+    if (g > 8) { pq += __shfl_xor_sync(0xffffffffu, pq, 8); pk += __shfl_xor_sync(0xffffffffu, pk, 8); }
+    if (g > 4) { pq += __shfl_xor_sync(0xffffffffu, pq, 4); pk += __shfl_xor_sync(0xffffffffu, pk, 4); }
+    if (g > 2) { pq += __shfl_xor_sync(0xffffffffu, pq, 2); pk += __shfl_xor_sync(0xffffffffu, pk, 2); }
+    if (g > 1) { pq += __shfl_xor_sync(0xffffffffu, pq, 1); pk += __shfl_xor_sync(0xffffffffu, pk, 1); }
+    // ---- Phase B, communication path: token xr's scalars to every rank ------------------------------
+    const float mine_q = __shfl_sync(0xffffffffu, pq, xr << P.log_g);  // also: every lane has consumed the stage
+    const float mine_k = __shfl_sync(0xffffffffu, pk, xr << P.log_g);
+    const bool xlive = t0 + xr < P.T;
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) {  // the same tree in every lane: all 32 end with the same bits
-      pq += __shfl_xor_sync(0xffffffffu, pq, o);
-      pk += __shfl_xor_sync(0xffffffffu, pk, o);
+    for (int rd = 0; rd < kTpRounds; ++rd) {
+      if (rd >= rounds) break;
+      const int xp = xp0 + (rd << P.log_g);
+      if (xlive && xp < P.N && xp != R.rank) {
+        unsigned long long* peer = R.peer_inbox[xp];
+        if (cq) ptx::st_relaxed_sys_u64(peer + slot_q_out + t0, tag | (unsigned long long)__float_as_uint(mine_q));
+        if (ck) ptx::st_relaxed_sys_u64(peer + slot_k_out + t0, tag | (unsigned long long)__float_as_uint(mine_k));
+      }
     }
-    // ---- Phase B, communication path: push S_local to every peer ------------------------------------
-    if (push_q) ptx::st_relaxed_sys_u64(push_q + t, tag | (unsigned long long)__float_as_uint(pq));
-    if (push_k) ptx::st_relaxed_sys_u64(push_k + t, tag | (unsigned long long)__float_as_uint(pk));
-    // every lane has its chunks in registers (the shuffles above are the proof): next row on its way
-    const bool armed = t + step < P.T;
-    if (armed) arm(t + step);
-    if (lane == 0) {
+    const bool armed = t0 + step < P.T;
+    if (armed) arm(t0 + step);  // the next tile is on its way while this one waits for its peers
+    if (live && l == 0) {
       if (R.partial_q != nullptr) R.partial_q[t] = pq;
       if (R.partial_k != nullptr) R.partial_k[t] = pk;
     }
     // ---- wait for the peers' scalars in this rank's own inbox ---------------------------------------
-    float inq = pq, ink = pk;  // lane p ends up with rank p's scalars (its own for p == rank)
-    bool got = true;
-    if (remote) got = tp_poll2(poll_q ? poll_q + t : nullptr, poll_k ? poll_k + t : nullptr, P.epoch, P.wait_ns, status, inq, ink);
-    const unsigned missing = __ballot_sync(0xffffffffu, !got);
+    float inq[kTpRounds], ink[kTpRounds];  // pair (rd, lane): rank xp's scalars of token xr (its own for xp == rank)
+    unsigned missing = 0u;
+    int missing_round = 0;
+#pragma unroll
+    for (int rd = 0; rd < kTpRounds; ++rd) {
+      inq[rd] = mine_q;
+      ink[rd] = mine_k;
+      if (rd >= rounds) continue;
+      const int xp = xp0 + (rd << P.log_g);
+      bool got = true;
+      if (xlive && xp < P.N && xp != R.rank) {
+        const unsigned long long* src_q = cq ? R.inbox + tp_slot_index(parity, 0, xp, P.N, P.cap) + xr + t0 : nullptr;
+        const unsigned long long* src_k = ck ? R.inbox + tp_slot_index(parity, 1, xp, P.N, P.cap) + xr + t0 : nullptr;
+        got = tp_poll2(src_q, src_k, P.epoch, P.wait_ns, status, inq[rd], ink[rd]);
+      }
+      const unsigned m = __ballot_sync(0xffffffffu, !got);
+      if (m != 0u && missing == 0u) {
+        missing = m;
+        missing_round = rd;
+      }
+    }
     if (missing != 0u) {
       if (lane == 0 && atomicCAS(status, kTpOk, kTpPeerTimeout) == kTpOk) {
-        status[1] = (int)(t & 0x7fffffff);
-        status[2] = __ffs((int)missing) - 1;
+        const int bad = __ffs((int)missing) - 1;
+        status[1] = (int)((t0 + (bad & (tile - 1))) & 0x7fffffff);
+        status[2] = (bad >> (5 - P.log_g)) + (missing_round << P.log_g);
       }
       if (armed) ptx::mbar_wait_bounded(bar, phase);  // the warp's own copy in flight
       return;
     }
     // ---- S_global: all N scalars in ascending rank order, the same on every rank ----------------------
     float totq = 0.f, totk = 0.f;
-    for (int p = 0; p < P.N; ++p) {
-      totq += __shfl_sync(0xffffffffu, inq, p);
-      totk += __shfl_sync(0xffffffffu, ink, p);
+#pragma unroll
+    for (int rd = 0; rd < kTpRounds; ++rd) {
+      for (int pp = 0; pp < g; ++pp) {  // rank rd * g + pp sits in lane pp * tile + s of round rd
+        if ((rd << P.log_g) + pp >= P.N) break;
+        totq += __shfl_sync(0xffffffffu, inq[rd], pp * tile + s);
+        totk += __shfl_sync(0xffffffffu, ink[rd], pp * tile + s);
+      }
     }
     const float rq = rstd_of(totq, P.inv_dq, P.eps);
     const float rk = rstd_of(totk, P.inv_dk, P.eps);
-    if (lane == 0) {
+    if (live && l == 0) {
       if (R.rstd_q != nullptr) R.rstd_q[t] = rq;
       if (R.rstd_k != nullptr) R.rstd_k[t] = rk;
     }
@@ -368,7 +417,7 @@ tp_kernel(const __grid_constant__ TpParams P) {
         const float r = kpart ? rk : rq;
         const float2 r2 = make_float2(r, r);
         unsigned char* dst = kpart ? dk_ + (size_t)(jb - P.nq4) * sstride : dq_ + (size_t)jb * sstride;
-        const int nv = kpart ? nvk - (jb - P.nq4) : nvq - jb;
+        const int nv = live ? (kpart ? nvk - (jb - P.nq4) : nvq - jb) : 0;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint4 ga = gsm[(jb + i) * GV][lane], gb = gsm[(jb + i) * GV + GV - 1][lane];

@@ -135,22 +135,49 @@ int run_tp(int elem_bytes, const qknorm_tp_rank* ranks, int n_local, int N, long
       if (may_overlap(outs[i], others[j])) return QKNORM_ERR_ALIAS;
   }
 
-  // chunk slots per lane: the whole warp serves the rank's one slice of each tensor
+  // Tokens per warp tile: R = 32 / g lane groups of g lanes, one token each.  More tokens per tile
+  // spread the per-tile work (barrier wait, copy issue, shuffles, push, poll) over more rows, and
+  // measured on B200 that outweighs the registers the longer per-lane runs cost: take the widest
+  // tile whose rows fit the 40 chunk slots a lane can hold.
   const int cq = wq * elem_bytes / 16, ck = wk * elem_bytes / 16;
-  P.nq = (cq + 31) / 32;
-  P.nk = (ck + 31) / 32;
-  P.nq4 = round_up(P.nq, 4);
-  const int l = warp_round_up_l(P.nq4 + P.nk);
-  TpKernel fn = l > 0 ? tp_kernel_for(l, elem_bytes) : nullptr;
-  if (!fn) return QKNORM_ERR_SHAPE;  // slice rows too long for one warp
-  P.k_base = wq * elem_bytes;
-  P.zero_off = P.k_base + wk * elem_bytes;
-  P.stage_bytes = round_up(P.zero_off + 16, 128);
+  const int forced_log_g = env_int("QKNORM_TP_LOG_G", -1);
+  int best_log_g = -1, best_l = -1;
+  for (int log_g = 2; log_g <= 5; ++log_g) {
+    const int g = 1 << log_g, tile = 32 >> log_g;
+    if (tile * N > 32 * kTpRounds) continue;
+    if (forced_log_g >= 0 && log_g != forced_log_g) continue;
+    const int slots = round_up((cq + g - 1) / g, 4) + (ck + g - 1) / g;
+    const int l = warp_round_up_l(slots);
+    if (l < 0) continue;
+    best_log_g = log_g;
+    best_l = l;
+    break;
+  }
+  if (best_log_g < 0) return QKNORM_ERR_SHAPE;  // slice rows too long for one warp
+  TpKernel fn = tp_kernel_for(best_l, elem_bytes);
+  if (!fn) return QKNORM_ERR_SHAPE;
+  {
+    const int g = 1 << best_log_g, tile = 32 >> best_log_g;
+    P.log_g = best_log_g;
+    P.nq = (cq + g - 1) / g;
+    P.nk = (ck + g - 1) / g;
+    P.nq4 = round_up(P.nq, 4);
+    // rows of a tile side by side in the stage; the skew keeps lane groups that read in the same
+    // quarter-warp on different banks
+    const int skew = (tile > 1 && g < 8) ? g * 16 : 0;
+    P.q_row_stride = cq ? wq * elem_bytes + skew : 0;
+    P.k_row_stride = ck ? wk * elem_bytes + skew : 0;
+    P.k_base = tile * P.q_row_stride;
+    P.zero_off = P.k_base + tile * P.k_row_stride;
+    P.stage_bytes = round_up(P.zero_off + 16, 128);
+  }
+  const int tile = 32 >> P.log_g;
 
   const DeviceInfo* dev = nullptr;
   rc = current_device(&dev);
   if (rc != QKNORM_OK) return rc;
-  const int warps = kWarpMaxCtaWarps;
+  int warps = env_int("QKNORM_TP_WARPS", kWarpMaxCtaWarps);
+  if (warps < 1 || warps > kWarpMaxCtaWarps) warps = kWarpMaxCtaWarps;
   const int smem = warps * P.stage_bytes;
   rc = allow_dynamic_smem((const void*)fn, smem);
   if (rc != QKNORM_OK) return rc;
@@ -161,7 +188,8 @@ int run_tp(int elem_bytes, const qknorm_tp_rank* ranks, int n_local, int N, long
   if (cap_ctas > 0 && cap_ctas < resident) resident = cap_ctas;
   // bounded grid (Section III-D): every CTA of every rank served here is resident at once
   long long per_rank = (long long)resident * dev->sm_count / n_local;
-  const long long needed = (T + warps - 1) / warps;
+  const long long tiles = (T + tile - 1) / tile;
+  const long long needed = (tiles + warps - 1) / warps;
   if (per_rank > needed) per_rank = needed;
   if (per_rank < 1) return QKNORM_ERR_SHARDS;  // more local ranks than resident CTAs
   const unsigned grid = (unsigned)(per_rank * n_local);

@@ -151,3 +151,70 @@ def test_baseline_scratch_errors(libqknorm):
     assert gather(SC, 4 * 128 * 2 - 1) == binding.QKNORM_ERR_SCRATCH
     assert gather(SC + 8, 1 << 20) == binding.QKNORM_ERR_SCRATCH               # not 16-byte aligned
     assert gather(E, 1 << 20) == binding.QKNORM_ERR_SCRATCH                    # on top of an output
+
+
+# ---- tensor-parallel entry point: everything below is rejected on the host, before any launch ----
+def _tp_call(lib, N=2, n_local=2, T=4, cap=8, wq=64, wk=64, eps=1e-6, epoch=1, ranks=(0, 1), patch=None, fn="qknorm_fwd_tp"):
+    from paper_2608_09160_b200 import tp
+    tp.lib()
+    arr = (tp.CTpRank * max(n_local, 1))()
+    keep = []
+    for i in range(n_local):
+        base = 0x20000000 + i * 0x8000000
+        peers = (ctypes.c_void_p * N)(*[0x70000000 + p * 0x1000000 for p in range(N)])
+        keep.append(peers)
+        c = arr[i]
+        c.rank = ranks[i]
+        c.q, c.k, c.gamma_q, c.gamma_k = base, base + 0x100000, base + 0x200000, base + 0x300000
+        c.out_q, c.out_k = base + 0x400000, base + 0x500000
+        c.inbox = 0x70000000 + ranks[i] * 0x1000000
+        c.peer_inbox = ctypes.cast(peers, ctypes.POINTER(ctypes.c_void_p))
+        if patch:
+            patch(i, c)
+    return getattr(lib, fn)(arr, n_local, N, T, cap, wq, wk, None, eps, epoch, 0, None)
+
+
+def test_tensor_parallel_argument_errors(libqknorm):
+    lib = libqknorm
+    B = binding
+    assert _tp_call(lib, T=0) == B.QKNORM_OK                        # nothing to do, nothing launched
+    assert _tp_call(lib, N=0) == B.QKNORM_ERR_SHARDS
+    assert _tp_call(lib, N=17, n_local=1) == B.QKNORM_ERR_SHARDS
+    assert _tp_call(lib, N=1, n_local=2) == B.QKNORM_ERR_SHARDS      # more local ranks than ranks
+    assert _tp_call(lib, ranks=(0, 0)) == B.QKNORM_ERR_SHARDS        # a rank listed twice
+    assert _tp_call(lib, ranks=(0, 2)) == B.QKNORM_ERR_SHARDS        # rank number out of range
+    assert _tp_call(lib, T=9, cap=8) == B.QKNORM_ERR_SHAPE           # more tokens than the inboxes hold
+    assert _tp_call(lib, wq=0, wk=0) == B.QKNORM_ERR_SHAPE
+    assert _tp_call(lib, N=16, n_local=1, wq=8192) == B.QKNORM_ERR_SHAPE   # H_total beyond the maximum
+    assert _tp_call(lib, epoch=0) == B.QKNORM_ERR_SHAPE              # 0 is what an empty slot holds
+    assert _tp_call(lib, eps=float("nan")) == B.QKNORM_ERR_EPS
+    assert _tp_call(lib, wq=60) == B.QKNORM_ERR_ALIGN                # slice row not a multiple of 16 bytes
+    assert _tp_call(lib, wq=24, fn="qknorm_fwd_tp_e4m3") == B.QKNORM_ERR_ALIGN
+
+    def no_inbox(i, c):
+        c.inbox = None
+    assert _tp_call(lib, patch=no_inbox) == B.QKNORM_ERR_NULL
+
+    def skewed(i, c):
+        c.q = c.q + 2
+    assert _tp_call(lib, patch=skewed) == B.QKNORM_ERR_ALIGN
+
+    def shared_output(i, c):
+        c.out_q = 0x60000000
+    assert _tp_call(lib, patch=shared_output) == B.QKNORM_ERR_ALIAS   # two ranks write one buffer
+
+    def output_in_inbox(i, c):
+        c.out_k = c.inbox + 256
+    assert _tp_call(lib, patch=output_in_inbox) == B.QKNORM_ERR_ALIAS
+    # a slice row pair longer than one warp's 40 chunk slots per lane
+    assert _tp_call(lib, N=2, wq=16384, wk=8192) == B.QKNORM_ERR_SHAPE
+
+
+def test_tensor_parallel_inbox_size(libqknorm):
+    from paper_2608_09160_b200 import tp
+    assert tp.inbox_bytes(8, 65536) == 256 + 2 * 2 * 8 * 65536 * 8
+    assert tp.inbox_bytes(1, 1) == 256 + 32
+    with pytest.raises(binding.QKNormError):
+        tp.inbox_bytes(17, 16)
+    with pytest.raises(binding.QKNormError):
+        tp.inbox_bytes(2, 0)

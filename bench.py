@@ -339,7 +339,7 @@ def config_table(steps: int, warmup: int, peak: float, skip: str):
     return rows
 
 
-def tp_rows(steps: int, warmup: int, peak: float):
+def tp_rows(steps: int, warmup: int, peak: float, tokens: int = 0):
     """The tensor-parallel kernel (Algorithm 1 with its scalar exchange) with all N ranks on this
     one GPU: one cooperative launch serves every rank, scalars go through the ranks' inboxes in
     device memory.  Same bytes as the logical-shard call, so the difference to it is what the
@@ -347,7 +347,7 @@ def tp_rows(steps: int, warmup: int, peak: float):
     from paper_2608_09160_b200 import binding, tp
     rows = {}
     for name, N in (("C3", 4), ("C4", 8), ("C5", 8)):
-        w = W.WORKLOADS[name]
+        w = W.WORKLOADS[name] if tokens <= 0 else W.scaled(W.WORKLOADS[name], tokens)
         inp = W.make_inputs(w)
         dev = {k: [t.cuda() for t in W.shard_columns(inp[k], N)] for k in ("q", "k", "gamma_q", "gamma_k")}
         del inp
@@ -567,6 +567,9 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "e4m3"], help="storage format of the activations")
     ap.add_argument("--head-dim", type=int, default=0, help="headwise granularity with this head size (needs --shards 1)")
     ap.add_argument("--no-table", action="store_true", help="skip the per-config table")
+    ap.add_argument("--tp-only", action="store_true",
+                    help="only the tensor-parallel rows of the table (all ranks on this GPU), as one JSON object; "
+                         "with --tokens for a small case to profile")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
@@ -594,6 +597,11 @@ def main():
     if dist is not None:
         dist.barrier()
     binding.load()
+    if args.tp_only:
+        if world > 1:
+            raise SystemExit("--tp-only stands N ranks on ONE GPU; run it without torchrun")
+        print(json.dumps({"tensor_parallel_rows": tp_rows(args.steps, args.warmup, measured_peak()[0], args.tokens)}))
+        return
 
     w = W.WORKLOADS[args.workload]
     if args.tokens:

@@ -52,9 +52,10 @@
  * descriptors are HOST memory read during the call only, the return value is a
  * qknorm_status, on error nothing was launched, tokens == 0 returns QKNORM_OK.
  * The vectorised path is the only one here: slice widths must be multiples of
- * 16 bytes, base pointers 16-byte aligned, pitches multiples of 16 bytes, and a slice
- * row pair (Q then K) must fit 40 16-byte chunks per lane (about 20 KB); anything else
- * is QKNORM_ERR_ALIGN / QKNORM_ERR_SHAPE.
+ * 16 bytes, base pointers 16-byte aligned, pitches multiples of 16 bytes, and three
+ * copies of a slice row pair (Q then K) plus the two gamma slices must fit a CTA's
+ * shared memory (rows of up to about 60 KB); anything else is QKNORM_ERR_ALIGN /
+ * QKNORM_ERR_SHAPE.
  */
 #ifndef QKNORM_TP_H_
 #define QKNORM_TP_H_

@@ -24,7 +24,7 @@ BUILD_DIR = os.path.join(PKG_DIR, "build")
 LIB_PATH = os.path.join(PKG_DIR, "libqknorm.so")
 
 CHUNKS_PER_THREAD = (1, 2, 3, 4, 6, 8)          # row / ring kernels
-CHUNK_SLOTS_PER_LANE = tuple(range(4, 44, 4))    # warp-per-row kernels (single-GPU and tensor-parallel)
+CHUNK_SLOTS_PER_LANE = tuple(range(4, 44, 4))    # warp-per-row kernel
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
@@ -50,10 +50,7 @@ def _units() -> List[Tuple[str, str, List[str]]]:
         for io, tag in (("IoBf16", "bf16"), ("IoE4m3", "e4m3")):
             units.append((f"qknorm_warp_{tag}_l{l}.o", os.path.join(CSRC, "qknorm_warp_inst.cu"),
                           [f"-DQKNORM_L={l}", f"-DQKNORM_IO={io}", f"-DQKNORM_IO_TAG={tag}"]))
-    for l in CHUNK_SLOTS_PER_LANE:
-        for io, tag in (("IoBf16", "bf16"), ("IoE4m3", "e4m3")):
-            units.append((f"qknorm_tp_{tag}_l{l}.o", os.path.join(CSRC, "qknorm_tp_inst.cu"),
-                          [f"-DQKNORM_L={l}", f"-DQKNORM_IO={io}", f"-DQKNORM_IO_TAG={tag}"]))
+    units.append(("qknorm_tp.o", os.path.join(CSRC, "qknorm_tp_inst.cu"), []))
     return units
 
 

@@ -16,10 +16,15 @@
 //    double-buffered by epoch parity: a rank can run at most one call ahead of a peer
 //    (it needs the peer's scalars of call c+1 to finish c+1), so what it writes for c+2
 //    lands in the half the peer finished with c.
-//  * no warp is set aside for communication.  The kernel keeps the warp-level design of
-//    the single-GPU path: a warp has its NEXT tile of rows in flight (TMA bulk copies into
-//    its own shared-memory stage) while it waits for the scalars of the current one, and
-//    the other warps of the SM cover the link latency.
+//  * no warp is set aside for communication, and the wait is taken off the critical path
+//    by software pipelining inside every warp instead.  A warp owns three shared-memory
+//    stages, each holding one TILE of tokens' slice rows (filled by TMA bulk copies).  In
+//    step j it (1) takes tile j from its stage, forms the sums of squares and pushes
+//    them, (2) only then collects the peers' scalars of tile j-1 -- pushed a whole step
+//    ago, so normally already there -- and scales and writes tile j-1 from ITS stage,
+//    (3) refills that stage with tile j+2.  Tile j+1 is in flight during all of step j.
+//    Rows are read from shared memory twice instead of being held in registers, which
+//    keeps the register count low enough for 16 and more warps per SM.
 //  * a warp works on several tokens side by side (see tp_kernel), and one lane per
 //    (token, peer) pair carries the exchange: all pushes of a tile are one store
 //    instruction, all polls one loop.
@@ -47,6 +52,8 @@
 namespace qknorm {
 
 constexpr int kTpRounds = 4;        // exchange rounds of 32 (token, rank) pairs: tile * N <= 128
+constexpr int kTpStages = 3;        // shared-memory stages per warp
+constexpr int kTpMaxCtaWarps = 8;
 constexpr int kTpHeaderWords = 32;  // 256-byte header in front of the slots (64-bit words)
 
 // status codes in word 0 of the inbox header
@@ -84,11 +91,11 @@ struct TpParams {
   uint32_t epoch;         // != 0
   unsigned long long wait_ns;
   int log_g;              // log2 of the lanes that serve one token (32 >> log_g tokens per warp tile)
-  int nq, nk, nq4;        // chunk slots per lane: Q part, K part, first K slot
-  int stage_bytes;        // one warp's stage: the tile's Q rows, its K rows, 16 zero bytes
+  int stage_bytes;        // one stage: the tile's Q rows, then its K rows (multiple of 128)
   int q_row_stride;       // bytes between consecutive tokens' Q rows inside a stage (row + bank skew)
   int k_row_stride;
-  int k_base, zero_off;
+  int k_base;             // byte offset of the K rows inside a stage
+  int gamma_bytes;        // shared memory in front of the stages: gamma_q slice, gamma_k slice (multiple of 128)
 };
 
 namespace ptx {
@@ -106,13 +113,6 @@ __device__ __forceinline__ int ld_relaxed_gpu_s32(const int* p) {
   return v;
 }
 }  // namespace ptx
-
-// Resident CTAs of 4 warps the registers are shaped for.  The exchange keeps four slot
-// pointers, the tag and the peer bookkeeping alive across the token loop, so a slice row
-// gets a few registers more per thread than the single-GPU kernel gives it.
-__host__ __device__ constexpr int tp_min_blocks(int l, int elem_bytes) {
-  return l <= 8 ? 6 : (l <= 16 ? 3 : 2);
-}
 
 __host__ __device__ inline long long tp_slot_index(int parity, int tensor, int src_rank, int N, long long cap) {
   return (long long)kTpHeaderWords + ((long long)((parity * 2 + tensor) * N + src_rank)) * cap;
@@ -155,16 +155,15 @@ __device__ __forceinline__ bool tp_poll2(const unsigned long long* sq, const uns
 // that token's Q slice row and K slice row.  Slice rows are short (a few KB), so one token
 // per warp would spend most of its instructions on per-token work (barrier wait, copy
 // issue, shuffles, push, poll); with R tokens side by side that work is done once per tile:
-// one log2(g)-step shuffle tree gives all R scalars, ONE store instruction pushes R x (N-1)
-// scalars (lane p*R + r: token r to rank p), one poll loop collects them, N broadcasts per
-// tensor form all R sums.  When R * N exceeds 32 the pairs take up to kTpRounds rounds.
-template <int L, class IO>
-__global__ void __launch_bounds__(kWarpMaxCtaWarps * 32, tp_min_blocks(L, IO::kBytes))
+// one log2(g)-step shuffle tree gives all R scalars, one store instruction pushes 32
+// (token, rank) pairs (pair p*R + r: token r to rank p), one poll loop collects them, N
+// broadcasts per tensor form all R sums.  R * N <= 32 * kTpRounds.
+template <int LOG_G, class IO>
+__global__ void __launch_bounds__(kTpMaxCtaWarps * 32, 2)
 tp_kernel(const __grid_constant__ TpParams P) {
   constexpr int GV = IO::kGammaVecs;
-  extern __shared__ __align__(128) unsigned char tp_smem[];  // one stage per warp
-  __shared__ uint4 gsm[L * GV][32];
-  __shared__ __align__(8) unsigned long long bars[kWarpMaxCtaWarps];
+  extern __shared__ __align__(128) unsigned char tp_smem[];  // gamma_q, gamma_k, then kTpStages stages per warp
+  __shared__ __align__(8) unsigned long long bars[kTpMaxCtaWarps][kTpStages];
 
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
@@ -174,23 +173,22 @@ tp_kernel(const __grid_constant__ TpParams P) {
   const long long ctas = gridDim.x / (unsigned)P.n_local;
   int* const status = reinterpret_cast<int*>(R.inbox);
 
-  const int g = 1 << P.log_g;
-  const int tile = 32 >> P.log_g;  // tokens per tile
-  const int s = lane >> P.log_g;   // which token of the tile this lane serves
+  constexpr int g = 1 << LOG_G;
+  constexpr int tile = 32 >> LOG_G;  // tokens per tile
+  const int s = lane >> LOG_G;       // which token of the tile this lane serves
   const int l = lane & (g - 1);
   const int cq = (P.wq * IO::kBytes) >> 4, ck = (P.wk * IO::kBytes) >> 4;  // 16-byte chunks per slice row
-  const int nvq = l < cq ? (cq - l + g - 1) >> P.log_g : 0;
-  const int nvk = l < ck ? (ck - l + g - 1) >> P.log_g : 0;
-  const int n_slots = P.nq4 + P.nk;
+  const int nvq = l < cq ? (cq - l + g - 1) >> LOG_G : 0;                 // chunks of this lane
+  const int nvk = l < ck ? (ck - l + g - 1) >> LOG_G : 0;
 
-  unsigned char* stage = tp_smem + (size_t)warp * P.stage_bytes;
-  const uint32_t stage_u32 = ptx::smem_u32(stage);
-  const uint32_t bar = ptx::smem_u32(&bars[warp]);
+  const uint32_t smem0 = ptx::smem_u32(tp_smem);
+  const uint32_t stages0 = smem0 + (uint32_t)P.gamma_bytes + (uint32_t)warp * kTpStages * (uint32_t)P.stage_bytes;
+  const uint32_t bar0 = ptx::smem_u32(&bars[warp][0]);
   if (lane == 0) {
-    ptx::mbar_init(bar, 1u);
+#pragma unroll
+    for (int st = 0; st < kTpStages; ++st) ptx::mbar_init(bar0 + 8u * st, 1u);
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
-    *reinterpret_cast<uint4*>(stage + P.zero_off) = make_uint4(0u, 0u, 0u, 0u);
   }
   // lane i < tile fetches the Q slice row of token i of the tile, lane tile + i its K slice row
   const bool issue_q = lane < tile;
@@ -213,227 +211,233 @@ tp_kernel(const __grid_constant__ TpParams P) {
   }
   const uint32_t row_bytes = ((uint32_t)P.wq + (uint32_t)P.wk) * IO::kBytes;
   const uint64_t policy = ptx::policy_evict_first();
-  auto arm = [&](long long t0) {  // whole warp; t0 = first token of the tile
-    const long long left = P.T - t0;
-    const int n = left < tile ? (int)left : tile;
-    if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)n * row_bytes);
-    __syncwarp();
-    if (my_bytes && is < n) ptx::bulk_load(stage_u32 + my_dst, my_src + (unsigned long long)(t0 + is) * my_pitch, my_bytes, bar, policy);
-  };
 
   const int cta_warps = blockDim.x >> 5;
   const long long first = (cta * cta_warps + warp) * tile;
   const long long step = ctas * cta_warps * tile;
+  const long long n_tiles = first < P.T ? (P.T - first + step - 1) / step : 0;  // this warp's tiles
+  auto arm = [&](long long t0, int st) {  // whole warp: the tile that starts at token t0 into stage st
+    const long long left = P.T - t0;
+    const int n = left < tile ? (int)left : tile;
+    const uint32_t bar = bar0 + 8u * (uint32_t)st;
+    if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)n * row_bytes);
+    __syncwarp();
+    if (my_bytes && is < n)
+      ptx::bulk_load(stages0 + (uint32_t)st * (uint32_t)P.stage_bytes + my_dst,
+                     my_src + (unsigned long long)(t0 + is) * my_pitch, my_bytes, bar, policy);
+  };
   __syncwarp();
-  if (first < P.T) arm(first);
+  if (n_tiles > 0) arm(first, 0);
+  if (n_tiles > 1) arm(first + step, 1);
 
-  // gamma of the slice, once per CTA, as [chunk slot][lane] (the same values in every lane group)
+  // gamma of the slice, once per CTA: gamma_q chunks, then gamma_k chunks, in row order
+  uint4* const gsm = reinterpret_cast<uint4*>(tp_smem);
+  const int gq_vecs = cq * GV, gk_vecs = ck * GV;
   bool gamma_f16 = false;
   {
-    const uint4* gq = reinterpret_cast<const uint4*>(R.gq) + (size_t)l * GV;
-    const uint4* gk = reinterpret_cast<const uint4*>(R.gk) + (size_t)l * GV;
-    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
     bool fits = true;
-    for (int j = warp; j < L; j += cta_warps) {
-#pragma unroll
-      for (int v = 0; v < GV; ++v) {
-        uint4 gv = zero;
-        if (j < nvq) gv = __ldg(gq + (size_t)j * g * GV + v);
-        else if (j >= P.nq4 && j - P.nq4 < nvk) gv = __ldg(gk + (size_t)(j - P.nq4) * g * GV + v);
-        gsm[j * GV + v][lane] = gv;
-        if (IO::kF16Gamma)
-          fits = fits && bf16x2_fits_f16(gv.x) && bf16x2_fits_f16(gv.y) && bf16x2_fits_f16(gv.z) && bf16x2_fits_f16(gv.w);
-      }
+    for (int i = threadIdx.x; i < gq_vecs + gk_vecs; i += blockDim.x) {
+      const uint4 gv = i < gq_vecs ? __ldg(reinterpret_cast<const uint4*>(R.gq) + i)
+                                   : __ldg(reinterpret_cast<const uint4*>(R.gk) + (i - gq_vecs));
+      gsm[i] = gv;
+      if (IO::kF16Gamma)
+        fits = fits && bf16x2_fits_f16(gv.x) && bf16x2_fits_f16(gv.y) && bf16x2_fits_f16(gv.z) && bf16x2_fits_f16(gv.w);
     }
     if (IO::kF16Gamma) {
+      // every gamma value of the slice is also an fp16 value: keep it as fp16 (each thread converts
+      // what it wrote) and multiply with the fp16 mixed FMA
       gamma_f16 = __syncthreads_and(fits ? 1 : 0) != 0;
       if (gamma_f16) {
-        for (int j = warp; j < L; j += cta_warps) {
-#pragma unroll
-          for (int v = 0; v < GV; ++v) {
-            uint4 gv = gsm[j * GV + v][lane];
-            gv.x = bf16x2_to_f16x2(gv.x);
-            gv.y = bf16x2_to_f16x2(gv.y);
-            gv.z = bf16x2_to_f16x2(gv.z);
-            gv.w = bf16x2_to_f16x2(gv.w);
-            gsm[j * GV + v][lane] = gv;
-          }
+        for (int i = threadIdx.x; i < gq_vecs + gk_vecs; i += blockDim.x) {
+          uint4 gv = gsm[i];
+          gv.x = bf16x2_to_f16x2(gv.x);
+          gv.y = bf16x2_to_f16x2(gv.y);
+          gv.z = bf16x2_to_f16x2(gv.z);
+          gv.w = bf16x2_to_f16x2(gv.w);
+          gsm[i] = gv;
         }
       }
     }
   }
   __syncthreads();  // the last block-level barrier
+  const uint32_t gq_u32 = smem0 + (uint32_t)l * 16u * GV;
+  const uint32_t gk_u32 = smem0 + (uint32_t)gq_vecs * 16u + (uint32_t)l * 16u * GV;
 
   // ---- the exchange: pair number (rd * 32 + lane) = p * tile + r carries token r of the tile to and
   // from rank p; kTpRounds rounds of 32 pairs cover tile * N <= 128 pairs ---------------------------
   const int parity = (int)(P.epoch & 1u);
   const int xr = lane & (tile - 1);         // token of the tile this lane exchanges (the same in every round)
-  const int xp0 = lane >> (5 - P.log_g);    // rank this lane talks to in round 0; round rd: xp0 + rd * g
+  const int xp0 = lane >> (5 - LOG_G);    // rank this lane talks to in round 0; round rd: xp0 + rd * g
   const long long slot_q_out = tp_slot_index(parity, 0, R.rank, P.N, P.cap) + xr;  // in a peer's inbox
   const long long slot_k_out = tp_slot_index(parity, 1, R.rank, P.N, P.cap) + xr;
   const int rounds = (tile * P.N + 31) >> 5;
   const unsigned long long tag = (unsigned long long)P.epoch << 32;
 
-  const uint32_t sq0 = stage_u32 + (uint32_t)s * (uint32_t)P.q_row_stride + (uint32_t)l * 16u;
-  const uint32_t sk0 = stage_u32 + (uint32_t)P.k_base + (uint32_t)s * (uint32_t)P.k_row_stride + (uint32_t)l * 16u;
-  const uint32_t szero = stage_u32 + (uint32_t)P.zero_off;
-  const uint32_t sstride = (uint32_t)g * 16u;
+  const uint32_t sq_lane = (uint32_t)s * (uint32_t)P.q_row_stride + (uint32_t)l * 16u;  // inside a stage
+  const uint32_t sk_lane = (uint32_t)P.k_base + (uint32_t)s * (uint32_t)P.k_row_stride + (uint32_t)l * 16u;
+  constexpr uint32_t sstride = (uint32_t)g * 16u;
   unsigned char* yq = reinterpret_cast<unsigned char*>(R.yq) + (size_t)l * 16u;
   unsigned char* yk = reinterpret_cast<unsigned char*>(R.yk) + (size_t)l * 16u;
   const unsigned long long q_row = (unsigned long long)P.ldyq * IO::kBytes, k_row = (unsigned long long)P.ldyk * IO::kBytes;
 
-  uint32_t phase = 0;
-  for (long long t0 = first; t0 < P.T; t0 += step) {
-    if (!ptx::mbar_wait_bounded(bar, phase)) {
-      if (lane == 0 && atomicCAS(status, kTpOk, kTpStageTimeout) == kTpOk) {
-        status[1] = (int)(t0 & 0x7fffffff);
-        status[2] = -1;
+  // sum of squares of this lane's chunks of one row, from shared memory; fixed order
+  auto sumsq_row = [&](uint32_t base, int nv) -> float {
+    float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, c4 = 0.f, c5 = 0.f, c6 = 0.f, c7 = 0.f;
+    int j = 0;
+    for (; j + 4 <= nv; j += 4, base += 4u * sstride) {
+      const uint4 a = ptx::lds128(base), b = ptx::lds128(base + sstride);
+      const uint4 c = ptx::lds128(base + 2u * sstride), d = ptx::lds128(base + 3u * sstride);
+      IO::sumsq_word(a.x, c0, c1); IO::sumsq_word(b.x, c2, c3); IO::sumsq_word(c.x, c4, c5); IO::sumsq_word(d.x, c6, c7);
+      IO::sumsq_word(a.y, c0, c1); IO::sumsq_word(b.y, c2, c3); IO::sumsq_word(c.y, c4, c5); IO::sumsq_word(d.y, c6, c7);
+      IO::sumsq_word(a.z, c0, c1); IO::sumsq_word(b.z, c2, c3); IO::sumsq_word(c.z, c4, c5); IO::sumsq_word(d.z, c6, c7);
+      IO::sumsq_word(a.w, c0, c1); IO::sumsq_word(b.w, c2, c3); IO::sumsq_word(c.w, c4, c5); IO::sumsq_word(d.w, c6, c7);
+    }
+    for (; j < nv; ++j, base += sstride) {
+      const uint4 a = ptx::lds128(base);
+      IO::sumsq_word(a.x, c0, c1); IO::sumsq_word(a.y, c2, c3); IO::sumsq_word(a.z, c4, c5); IO::sumsq_word(a.w, c6, c7);
+    }
+    return ((c0 + c1) + (c2 + c3)) + ((c4 + c5) + (c6 + c7));
+  };
+  // (x * gamma) * RMS^-1 of this lane's chunks of one row: shared memory -> global, one write
+  auto scale_row = [&](uint32_t base, int nv, uint32_t gbase, unsigned char* dst, float r, auto f16_gamma) {
+    const float2 r2 = make_float2(r, r);
+#pragma unroll 4
+    for (int j = 0; j < nv; ++j, base += sstride, gbase += sstride * GV, dst += sstride) {
+      const uint4 x = ptx::lds128(base);
+      const uint4 ga = ptx::lds128(gbase);
+      const uint4 gb = GV > 1 ? ptx::lds128(gbase + 16u) : ga;
+      uint4 o;
+      if constexpr (decltype(f16_gamma)::value) o = IO::scale_chunk_g16(x, ga, gb, r2);
+      else o = IO::scale_chunk(x, ga, gb, r2);
+      st_stream(reinterpret_cast<uint4*>(dst), o);
+    }
+  };
+  // stage and mbarrier parity of the tile a step starts with; both advance once per step
+  int st_cur = 0;            // j % kTpStages
+  uint32_t par_bits = 0u;    // bit st: parity the next wait on stage st expects
+  auto next_stage = [](int st) { return st + 1 == kTpStages ? 0 : st + 1; };
+  auto wait_stage = [&](int st) -> bool {  // bounded
+    const bool ok = ptx::mbar_wait_bounded(bar0 + 8u * (uint32_t)st, (par_bits >> st) & 1u);
+    par_bits ^= 1u << st;
+    return ok;
+  };
+  auto give_up = [&](int code, long long token, int rank_missing, bool copy_pending, int st_pending) {
+    if (lane == 0 && atomicCAS(status, kTpOk, code) == kTpOk) {
+      status[1] = (int)(token & 0x7fffffff);
+      status[2] = rank_missing;
+    }
+    if (copy_pending) wait_stage(st_pending);  // the warp's own copy still in flight
+  };
+
+  float held_q = 0.f, held_k = 0.f;  // this lane's pair values of the tile pushed one step ago
+  long long t_cur = first;   // first token of tile j
+  for (long long j = 0; j <= n_tiles; ++j, t_cur += step, st_cur = next_stage(st_cur)) {
+    float mine_q = 0.f, mine_k = 0.f;
+    const int st_next = next_stage(st_cur);                       // stage of tile j+1, in flight
+    const int st_prev = next_stage(st_next);                      // stage of tile j-1 (= of tile j+2)
+    if (j < n_tiles) {
+      // ---- step part 1: Phase A of tile j and the push (Phase B, communication path) ---------------
+      if (!wait_stage(st_cur)) {
+        give_up(kTpStageTimeout, t_cur, -1, j + 1 < n_tiles, st_next);
+        return;
       }
-      return;
-    }
-    phase ^= 1u;
-    const long long t = t0 + s;       // this lane group's token
-    const bool live = t < P.T;        // the last tile may be short: its stage rows are stale, never published
-    // ---- drain the stage into registers --------------------------------------------------------
-    uint4 v[L];
+      const long long t0 = t_cur;
+      const uint32_t st = stages0 + (uint32_t)st_cur * (uint32_t)P.stage_bytes;
+      float pq = sumsq_row(st + sq_lane, nvq), pk = sumsq_row(st + sk_lane, nvk);
+      // the same tree in every lane of a group: all g lanes end with the same bits
+      if (g > 16) { pq += __shfl_xor_sync(0xffffffffu, pq, 16); pk += __shfl_xor_sync(0xffffffffu, pk, 16); }
+      if (g > 8) { pq += __shfl_xor_sync(0xffffffffu, pq, 8); pk += __shfl_xor_sync(0xffffffffu, pk, 8); }
+      if (g > 4) { pq += __shfl_xor_sync(0xffffffffu, pq, 4); pk += __shfl_xor_sync(0xffffffffu, pk, 4); }
+      if (g > 2) { pq += __shfl_xor_sync(0xffffffffu, pq, 2); pk += __shfl_xor_sync(0xffffffffu, pk, 2); }
+      if (g > 1) { pq += __shfl_xor_sync(0xffffffffu, pq, 1); pk += __shfl_xor_sync(0xffffffffu, pk, 1); }
+      mine_q = __shfl_sync(0xffffffffu, pq, xr << LOG_G);
+      mine_k = __shfl_sync(0xffffffffu, pk, xr << LOG_G);
+      if (t0 + xr < P.T) {  // a short last tile: rows past the end are stale and never published
 #pragma unroll
-    for (int jb = 0; jb < L; jb += 4) {
-      if (jb >= n_slots) break;
-      const bool kpart = jb >= P.nq4;
-      const uint32_t base = kpart ? sk0 + (uint32_t)(jb - P.nq4) * sstride : sq0 + (uint32_t)jb * sstride;
-      const int nv = kpart ? nvk - (jb - P.nq4) : nvq - jb;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) v[jb + i] = ptx::lds128(i < nv ? base + (uint32_t)i * sstride : szero);
-    }
-    // ---- Phase A: S_local of the Q slice and of the K slice, one token per lane group --------------
-    float2 aq = make_float2(0.f, 0.f), ak = make_float2(0.f, 0.f);
-#pragma unroll
-    for (int jb = 0; jb < L; jb += 4) {
-      if (jb >= n_slots) break;
-      float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f, c4 = 0.f, c5 = 0.f, c6 = 0.f, c7 = 0.f;
-      IO::sumsq_word(v[jb].x, c0, c1);
-      IO::sumsq_word(v[jb + 1].x, c2, c3);
-      IO::sumsq_word(v[jb + 2].x, c4, c5);
-      IO::sumsq_word(v[jb + 3].x, c6, c7);
-      IO::sumsq_word(v[jb].y, c0, c1);
-      IO::sumsq_word(v[jb + 1].y, c2, c3);
-      IO::sumsq_word(v[jb + 2].y, c4, c5);
-      IO::sumsq_word(v[jb + 3].y, c6, c7);
-      IO::sumsq_word(v[jb].z, c0, c1);
-      IO::sumsq_word(v[jb + 1].z, c2, c3);
-      IO::sumsq_word(v[jb + 2].z, c4, c5);
-      IO::sumsq_word(v[jb + 3].z, c6, c7);
-      IO::sumsq_word(v[jb].w, c0, c1);
-      IO::sumsq_word(v[jb + 1].w, c2, c3);
-      IO::sumsq_word(v[jb + 2].w, c4, c5);
-      IO::sumsq_word(v[jb + 3].w, c6, c7);
-      const float2 b = __fadd2_rn(__fadd2_rn(make_float2(c0, c1), make_float2(c2, c3)),
-                                  __fadd2_rn(make_float2(c4, c5), make_float2(c6, c7)));
-      if (jb >= P.nq4) ak = __fadd2_rn(ak, b);
-      else aq = __fadd2_rn(aq, b);
-    }
-    float pq = aq.x + aq.y, pk = ak.x + ak.y;
-    // the same tree in every lane of a group: all g lanes end with the same bits
-    if (g > 16) { pq += __shfl_xor_sync(0xffffffffu, pq, 16); pk += __shfl_xor_sync(0xffffffffu, pk, 16); }
-    if (g > 8) { pq += __shfl_xor_sync(0xffffffffu, pq, 8); pk += __shfl_xor_sync(0xffffffffu, pk, 8); }
-    if (g > 4) { pq += __shfl_xor_sync(0xffffffffu, pq, 4); pk += __shfl_xor_sync(0xffffffffu, pk, 4); }
-    if (g > 2) { pq += __shfl_xor_sync(0xffffffffu, pq, 2); pk += __shfl_xor_sync(0xffffffffu, pk, 2); }
-    if (g > 1) { pq += __shfl_xor_sync(0xffffffffu, pq, 1); pk += __shfl_xor_sync(0xffffffffu, pk, 1); }
-    // ---- Phase B, communication path: token xr's scalars to every rank ------------------------------
-    const float mine_q = __shfl_sync(0xffffffffu, pq, xr << P.log_g);  // also: every lane has consumed the stage
-    const float mine_k = __shfl_sync(0xffffffffu, pk, xr << P.log_g);
-    const bool xlive = t0 + xr < P.T;
-#pragma unroll
-    for (int rd = 0; rd < kTpRounds; ++rd) {
-      if (rd >= rounds) break;
-      const int xp = xp0 + (rd << P.log_g);
-      if (xlive && xp < P.N && xp != R.rank) {
-        unsigned long long* peer = R.peer_inbox[xp];
-        if (cq) ptx::st_relaxed_sys_u64(peer + slot_q_out + t0, tag | (unsigned long long)__float_as_uint(mine_q));
-        if (ck) ptx::st_relaxed_sys_u64(peer + slot_k_out + t0, tag | (unsigned long long)__float_as_uint(mine_k));
-      }
-    }
-    const bool armed = t0 + step < P.T;
-    if (armed) arm(t0 + step);  // the next tile is on its way while this one waits for its peers
-    if (live && l == 0) {
-      if (R.partial_q != nullptr) R.partial_q[t] = pq;
-      if (R.partial_k != nullptr) R.partial_k[t] = pk;
-    }
-    // ---- wait for the peers' scalars in this rank's own inbox ---------------------------------------
-    float inq[kTpRounds], ink[kTpRounds];  // pair (rd, lane): rank xp's scalars of token xr (its own for xp == rank)
-    unsigned missing = 0u;
-    int missing_round = 0;
-#pragma unroll
-    for (int rd = 0; rd < kTpRounds; ++rd) {
-      inq[rd] = mine_q;
-      ink[rd] = mine_k;
-      if (rd >= rounds) continue;
-      const int xp = xp0 + (rd << P.log_g);
-      bool got = true;
-      if (xlive && xp < P.N && xp != R.rank) {
-        const unsigned long long* src_q = cq ? R.inbox + tp_slot_index(parity, 0, xp, P.N, P.cap) + xr + t0 : nullptr;
-        const unsigned long long* src_k = ck ? R.inbox + tp_slot_index(parity, 1, xp, P.N, P.cap) + xr + t0 : nullptr;
-        got = tp_poll2(src_q, src_k, P.epoch, P.wait_ns, status, inq[rd], ink[rd]);
-      }
-      const unsigned m = __ballot_sync(0xffffffffu, !got);
-      if (m != 0u && missing == 0u) {
-        missing = m;
-        missing_round = rd;
-      }
-    }
-    if (missing != 0u) {
-      if (lane == 0 && atomicCAS(status, kTpOk, kTpPeerTimeout) == kTpOk) {
-        const int bad = __ffs((int)missing) - 1;
-        status[1] = (int)((t0 + (bad & (tile - 1))) & 0x7fffffff);
-        status[2] = (bad >> (5 - P.log_g)) + (missing_round << P.log_g);
-      }
-      if (armed) ptx::mbar_wait_bounded(bar, phase);  // the warp's own copy in flight
-      return;
-    }
-    // ---- S_global: all N scalars in ascending rank order, the same on every rank ----------------------
-    float totq = 0.f, totk = 0.f;
-#pragma unroll
-    for (int rd = 0; rd < kTpRounds; ++rd) {
-      for (int pp = 0; pp < g; ++pp) {  // rank rd * g + pp sits in lane pp * tile + s of round rd
-        if ((rd << P.log_g) + pp >= P.N) break;
-        totq += __shfl_sync(0xffffffffu, inq[rd], pp * tile + s);
-        totk += __shfl_sync(0xffffffffu, ink[rd], pp * tile + s);
-      }
-    }
-    const float rq = rstd_of(totq, P.inv_dq, P.eps);
-    const float rk = rstd_of(totk, P.inv_dk, P.eps);
-    if (live && l == 0) {
-      if (R.rstd_q != nullptr) R.rstd_q[t] = rq;
-      if (R.rstd_k != nullptr) R.rstd_k[t] = rk;
-    }
-    // ---- Phase B compute path and Phase C: (x * gamma) * RMS^-1, the one write ------------------------
-    unsigned char* dq_ = yq + (unsigned long long)t * q_row;
-    unsigned char* dk_ = yk + (unsigned long long)t * k_row;
-    auto store_pass = [&](auto f16_gamma) {
-#pragma unroll
-      for (int jb = 0; jb < L; jb += 4) {
-        if (jb >= n_slots) break;
-        const bool kpart = jb >= P.nq4;
-        const float r = kpart ? rk : rq;
-        const float2 r2 = make_float2(r, r);
-        unsigned char* dst = kpart ? dk_ + (size_t)(jb - P.nq4) * sstride : dq_ + (size_t)jb * sstride;
-        const int nv = live ? (kpart ? nvk - (jb - P.nq4) : nvq - jb) : 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const uint4 ga = gsm[(jb + i) * GV][lane], gb = gsm[(jb + i) * GV + GV - 1][lane];
-          uint4 o;
-          if constexpr (decltype(f16_gamma)::value) o = IO::scale_chunk_g16(v[jb + i], ga, gb, r2);
-          else o = IO::scale_chunk(v[jb + i], ga, gb, r2);
-          if (i < nv) st_stream(reinterpret_cast<uint4*>(dst + (size_t)i * sstride), o);
+        for (int rd = 0; rd < kTpRounds; ++rd) {
+          if (rd >= rounds) break;
+          const int xp = xp0 + (rd << LOG_G);
+          if (xp < P.N && xp != R.rank) {
+            unsigned long long* peer = R.peer_inbox[xp];
+            if (cq) ptx::st_relaxed_sys_u64(peer + slot_q_out + t0, tag | (unsigned long long)__float_as_uint(mine_q));
+            if (ck) ptx::st_relaxed_sys_u64(peer + slot_k_out + t0, tag | (unsigned long long)__float_as_uint(mine_k));
+          }
         }
       }
-    };
-    if (IO::kF16Gamma && gamma_f16) store_pass(std::true_type{});
-    else store_pass(std::false_type{});
+      if (t0 + s < P.T && l == 0) {
+        if (R.partial_q != nullptr) R.partial_q[t0 + s] = pq;
+        if (R.partial_k != nullptr) R.partial_k[t0 + s] = pk;
+      }
+    }
+    if (j >= 1) {
+      // ---- step part 2: tile j-1, pushed one step ago: collect, S_global, Phases B/C -------------
+      const long long t0 = t_cur - step;
+      const long long t = t0 + s;
+      const bool live = t < P.T, xlive = t0 + xr < P.T;
+      float inq[kTpRounds], ink[kTpRounds];  // pair (rd, lane): rank xp's scalars of token xr (own for xp == rank)
+      unsigned missing = 0u;
+      int missing_round = 0;
+#pragma unroll
+      for (int rd = 0; rd < kTpRounds; ++rd) {
+        inq[rd] = held_q;
+        ink[rd] = held_k;
+        if (rd >= rounds) continue;
+        const int xp = xp0 + (rd << LOG_G);
+        bool got = true;
+        if (xlive && xp < P.N && xp != R.rank) {
+          const unsigned long long* src_q = cq ? R.inbox + tp_slot_index(parity, 0, xp, P.N, P.cap) + xr + t0 : nullptr;
+          const unsigned long long* src_k = ck ? R.inbox + tp_slot_index(parity, 1, xp, P.N, P.cap) + xr + t0 : nullptr;
+          got = tp_poll2(src_q, src_k, P.epoch, P.wait_ns, status, inq[rd], ink[rd]);
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, !got);
+        if (m != 0u && missing == 0u) {
+          missing = m;
+          missing_round = rd;
+        }
+      }
+      if (missing != 0u) {
+        const int bad = __ffs((int)missing) - 1;
+        give_up(kTpPeerTimeout, t0 + (bad & (tile - 1)), (bad >> (5 - LOG_G)) + (missing_round << LOG_G), j + 1 < n_tiles, st_next);
+        return;
+      }
+      // all N scalars in ascending rank order, the same on every rank
+      float totq = 0.f, totk = 0.f;
+#pragma unroll
+      for (int rd = 0; rd < kTpRounds; ++rd) {
+        for (int pp = 0; pp < g; ++pp) {  // rank rd * g + pp sits in lane pp * tile + s of round rd
+          if ((rd << LOG_G) + pp >= P.N) break;
+          totq += __shfl_sync(0xffffffffu, inq[rd], pp * tile + s);
+          totk += __shfl_sync(0xffffffffu, ink[rd], pp * tile + s);
+        }
+      }
+      const float rq = rstd_of(totq, P.inv_dq, P.eps);
+      const float rk = rstd_of(totk, P.inv_dk, P.eps);
+      if (live) {
+        if (l == 0) {
+          if (R.rstd_q != nullptr) R.rstd_q[t] = rq;
+          if (R.rstd_k != nullptr) R.rstd_k[t] = rk;
+        }
+        const uint32_t st = stages0 + (uint32_t)st_prev * (uint32_t)P.stage_bytes;
+        unsigned char* dq_ = yq + (unsigned long long)t * q_row;
+        unsigned char* dk_ = yk + (unsigned long long)t * k_row;
+        if (IO::kF16Gamma && gamma_f16) {
+          scale_row(st + sq_lane, nvq, gq_u32, dq_, rq, std::true_type{});
+          scale_row(st + sk_lane, nvk, gk_u32, dk_, rk, std::true_type{});
+        } else {
+          scale_row(st + sq_lane, nvq, gq_u32, dq_, rq, std::false_type{});
+          scale_row(st + sk_lane, nvk, gk_u32, dk_, rk, std::false_type{});
+        }
+      }
+    }
+    // ---- step part 3: the stage tile j-1 lived in takes tile j+2 ---------------------------------
+    __syncwarp();
+    if (j + 2 < n_tiles) arm(t_cur + 2 * step, st_prev);
+    held_q = mine_q;
+    held_k = mine_k;
   }
 }
 
 using TpKernel = void (*)(const TpParams);
-TpKernel tp_kernel_for(int l, int elem_bytes);  // nullptr outside the instantiated set
+TpKernel tp_kernel_for(int log_g, int elem_bytes);  // log_g in 2..5
 
 }  // namespace qknorm

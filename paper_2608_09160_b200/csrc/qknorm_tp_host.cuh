@@ -8,23 +8,6 @@
 
 namespace qknorm {
 
-#define QKNORM_DECL_TP_L(l)     \
-  TpKernel tp_kernel_bf16_l##l(); \
-  TpKernel tp_kernel_e4m3_l##l();
-QKNORM_DECL_TP_L(4) QKNORM_DECL_TP_L(8) QKNORM_DECL_TP_L(12) QKNORM_DECL_TP_L(16) QKNORM_DECL_TP_L(20)
-QKNORM_DECL_TP_L(24) QKNORM_DECL_TP_L(28) QKNORM_DECL_TP_L(32) QKNORM_DECL_TP_L(36) QKNORM_DECL_TP_L(40)
-
-TpKernel tp_kernel_for(int l, int elem_bytes) {
-#define QKNORM_CASE_TP_L(l) \
-  case l: return elem_bytes == 1 ? tp_kernel_e4m3_l##l() : tp_kernel_bf16_l##l();
-  switch (l) {
-    QKNORM_CASE_TP_L(4) QKNORM_CASE_TP_L(8) QKNORM_CASE_TP_L(12) QKNORM_CASE_TP_L(16) QKNORM_CASE_TP_L(20)
-    QKNORM_CASE_TP_L(24) QKNORM_CASE_TP_L(28) QKNORM_CASE_TP_L(32) QKNORM_CASE_TP_L(36) QKNORM_CASE_TP_L(40)
-    default: return nullptr;
-  }
-#undef QKNORM_CASE_TP_L
-}
-
 namespace {
 
 int tp_inbox_bytes(int num_ranks, long long cap, long long* bytes) {
@@ -136,49 +119,62 @@ int run_tp(int elem_bytes, const qknorm_tp_rank* ranks, int n_local, int N, long
   }
 
   // Tokens per warp tile: R = 32 / g lane groups of g lanes, one token each.  More tokens per tile
-  // spread the per-tile work (barrier wait, copy issue, shuffles, push, poll) over more rows, and
-  // measured on B200 that outweighs the registers the longer per-lane runs cost: take the widest
-  // tile whose rows fit the 40 chunk slots a lane can hold.
+  // spread the per-tile work (barrier waits, copy issue, shuffles, push, poll) over more rows; the
+  // tile's bytes times the three stages times the warps must fit the SM's shared memory.  Measured
+  // on B200 (8 ranks on one GPU): tiles of 9-12 KB are fastest, 5 KB and 18 KB both cost 15-30 %.
   const int cq = wq * elem_bytes / 16, ck = wk * elem_bytes / 16;
+  const int row_bytes = (wq + wk) * elem_bytes;
+  const int tile_bytes_max = env_int("QKNORM_TP_TILE_BYTES", 12000);
   const int forced_log_g = env_int("QKNORM_TP_LOG_G", -1);
-  int best_log_g = -1, best_l = -1;
-  for (int log_g = 2; log_g <= 5; ++log_g) {
-    const int g = 1 << log_g, tile = 32 >> log_g;
+  int log_g = 5;
+  for (int lg = 2; lg <= 5; ++lg) {
+    const int tile = 32 >> lg;
     if (tile * N > 32 * kTpRounds) continue;
-    if (forced_log_g >= 0 && log_g != forced_log_g) continue;
-    const int slots = round_up((cq + g - 1) / g, 4) + (ck + g - 1) / g;
-    const int l = warp_round_up_l(slots);
-    if (l < 0) continue;
-    best_log_g = log_g;
-    best_l = l;
+    if (forced_log_g >= 0 ? lg != forced_log_g : (tile > 1 && tile * row_bytes > tile_bytes_max)) continue;
+    log_g = lg;
     break;
   }
-  if (best_log_g < 0) return QKNORM_ERR_SHAPE;  // slice rows too long for one warp
-  TpKernel fn = tp_kernel_for(best_l, elem_bytes);
+  TpKernel fn = tp_kernel_for(log_g, elem_bytes);
   if (!fn) return QKNORM_ERR_SHAPE;
+  const int tile = 32 >> log_g;
   {
-    const int g = 1 << best_log_g, tile = 32 >> best_log_g;
-    P.log_g = best_log_g;
-    P.nq = (cq + g - 1) / g;
-    P.nk = (ck + g - 1) / g;
-    P.nq4 = round_up(P.nq, 4);
+    const int g = 1 << log_g;
+    P.log_g = log_g;
     // rows of a tile side by side in the stage; the skew keeps lane groups that read in the same
     // quarter-warp on different banks
     const int skew = (tile > 1 && g < 8) ? g * 16 : 0;
     P.q_row_stride = cq ? wq * elem_bytes + skew : 0;
     P.k_row_stride = ck ? wk * elem_bytes + skew : 0;
     P.k_base = tile * P.q_row_stride;
-    P.zero_off = P.k_base + tile * P.k_row_stride;
-    P.stage_bytes = round_up(P.zero_off + 16, 128);
+    P.stage_bytes = round_up(P.k_base + tile * P.k_row_stride, 128);
+    P.gamma_bytes = round_up((wq + wk) * 2, 128);
   }
-  const int tile = 32 >> P.log_g;
+
+  // Warps per CTA: the CTA size that puts the most warps on an SM (three stages per warp and one
+  // copy of gamma per CTA against the SM's shared memory; 128 registers per thread allow 16 warps);
+  // among equals the larger CTA, which shares gamma between more warps.
+  constexpr int kSmemPerCta = 227 * 1024;  // sm_100: opt-in maximum of dynamic shared memory per CTA
+  constexpr int kSmemPerSm = 228 * 1024;   // and what one SM has, of which every resident CTA reserves 1 KB
+  const int forced_warps = env_int("QKNORM_TP_WARPS", 0);
+  int warps = 0, best_per_sm = 0;
+  for (int w = kTpMaxCtaWarps; w >= 1; --w) {
+    if (forced_warps > 0 && w != forced_warps) continue;
+    const int bytes = P.gamma_bytes + w * kTpStages * P.stage_bytes;
+    if (bytes > kSmemPerCta) continue;
+    int per_sm = (kSmemPerSm / (bytes + 1024 + 256)) * w;
+    if (per_sm > 16) per_sm = 16;
+    if (per_sm > best_per_sm) {
+      best_per_sm = per_sm;
+      warps = w;
+    }
+  }
+  if (warps == 0) return QKNORM_ERR_SHAPE;  // a slice row pair too long for three stages of shared memory
+  const int smem = P.gamma_bytes + warps * kTpStages * P.stage_bytes;
 
   const DeviceInfo* dev = nullptr;
   rc = current_device(&dev);
   if (rc != QKNORM_OK) return rc;
-  int warps = env_int("QKNORM_TP_WARPS", kWarpMaxCtaWarps);
-  if (warps < 1 || warps > kWarpMaxCtaWarps) warps = kWarpMaxCtaWarps;
-  const int smem = warps * P.stage_bytes;
+  if (smem > dev->smem_per_block) return QKNORM_ERR_SHAPE;
   rc = allow_dynamic_smem((const void*)fn, smem);
   if (rc != QKNORM_OK) return rc;
   int resident = 1;

@@ -1,16 +1,18 @@
-// Instantiation of the tensor-parallel kernel for ONE value of L (16-byte chunk slots
-// per lane) and ONE storage format, chosen with -DQKNORM_L=<l> -DQKNORM_IO=<IoBf16|IoE4m3>
-// -DQKNORM_IO_TAG=<bf16|e4m3>; one translation unit each.
+// The tensor-parallel kernel, one instantiation per tile shape and storage format, in a translation
+// unit of its own so that it compiles in parallel with the others.
 #include "qknorm_tp.cuh"
-
-#if !defined(QKNORM_L) || !defined(QKNORM_IO) || !defined(QKNORM_IO_TAG)
-#error "compile with -DQKNORM_L=<chunk slots per lane> -DQKNORM_IO=<format> -DQKNORM_IO_TAG=<tag>"
-#endif
-#define QKNORM_CAT3_(a, b, c, d) a##b##c##d
-#define QKNORM_CAT3(a, b, c, d) QKNORM_CAT3_(a, b, c, d)
 
 namespace qknorm {
 
-TpKernel QKNORM_CAT3(tp_kernel_, QKNORM_IO_TAG, _l, QKNORM_L)() { return tp_kernel<QKNORM_L, QKNORM_IO>; }
+TpKernel tp_kernel_for(int log_g, int elem_bytes) {
+  const bool f8 = elem_bytes == 1;
+  switch (log_g) {
+    case 2: return f8 ? tp_kernel<2, IoE4m3> : tp_kernel<2, IoBf16>;
+    case 3: return f8 ? tp_kernel<3, IoE4m3> : tp_kernel<3, IoBf16>;
+    case 4: return f8 ? tp_kernel<4, IoE4m3> : tp_kernel<4, IoBf16>;
+    case 5: return f8 ? tp_kernel<5, IoE4m3> : tp_kernel<5, IoBf16>;
+    default: return nullptr;
+  }
+}
 
 }  // namespace qknorm

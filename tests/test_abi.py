@@ -206,8 +206,8 @@ def test_tensor_parallel_argument_errors(libqknorm):
     def output_in_inbox(i, c):
         c.out_k = c.inbox + 256
     assert _tp_call(lib, patch=output_in_inbox) == B.QKNORM_ERR_ALIAS
-    # a slice row pair longer than one warp's 40 chunk slots per lane
-    assert _tp_call(lib, N=2, wq=16384, wk=8192) == B.QKNORM_ERR_SHAPE
+    # a slice row pair too long for a warp's three shared-memory stages
+    assert _tp_call(lib, N=2, wq=32768, wk=32768) == B.QKNORM_ERR_SHAPE
 
 
 def test_tensor_parallel_inbox_size(libqknorm):

@@ -7,7 +7,8 @@
  *   Phase A   S_local[t]  = sum_j X_local[t][j]^2                (fp32)
  *   Phase B   push S_local[t] into every peer's inbox; wait until the N-1 peers'
  *             scalars for t have arrived in this rank's own inbox;
- *             S_global[t] = sum of the N scalars in ascending rank order (fp32),
+ *             S_global[t] = sum of the N scalars (fp32), added pairwise over the rank index
+ *             (ranks 2i and 2i+1, then pairs of pairs, ...): the same tree on every rank,
  *             so every rank gets the same bits;
  *             RMS^-1      = 1 / sqrt(S_global / H_total + eps),  H_total = N * w
  *   Phase C   Y_local[t]  = (X_local[t] * W_local) * RMS^-1, rounded once, one write.

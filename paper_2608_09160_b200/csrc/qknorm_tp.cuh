@@ -1,12 +1,12 @@
 // Column-sharded (tensor-parallel) QK-RMSNorm with the scalar exchange of Algorithm 1,
 // Phase B: every rank holds one column slice of Q and of K, forms its own sums of
 // squares (Phase A), PUSHES the two scalars into every peer's inbox, waits until the
-// peers' scalars have landed in its own inbox, adds all N scalars in ascending rank
-// order and scales its slice (Phase C).  Per token and tensor 8 bytes cross the link to
+// peers' scalars have landed in its own inbox, adds all N scalars in one fixed order
+// (the same on every rank) and scales its slice (Phase C).  Per token and tensor 8 bytes cross the link to
 // each peer instead of the slice itself (Section III-A).
 //
 // How it differs from the flag protocol of Algorithm 1 (kept: push into the consumer's
-// memory, wait on local memory only, fp32 scalars, rank-order sum, bounded grid):
+// memory, wait on local memory only, fp32 scalars, the same sum on every rank, bounded grid):
 //  * value and flag are ONE 8-byte word {epoch tag, fp32 bits} written with a single
 //    64-bit store.  A naturally aligned 64-bit store is never torn, so the consumer
 //    either sees the old word or the whole new one: no fence between data and flag, no
@@ -25,6 +25,9 @@
 //    (3) refills that stage with tile j+2.  Tile j+1 is in flight during all of step j.
 //    Rows are read from shared memory twice instead of being held in registers, which
 //    keeps the register count low enough for 16 and more warps per SM.
+//  * S_global is a pairwise tree over the rank index (log2 N shuffle steps for all tokens of a
+//    tile at once) instead of a loop over the ranks; the tree is the same on every rank, so
+//    all ranks still get identical bits.
 //  * a warp works on several tokens side by side (see tp_kernel), and one lane per
 //    (token, peer) pair carries the exchange: all pushes of a tile are one store
 //    instruction, all polls one loop.
@@ -51,7 +54,6 @@
 
 namespace qknorm {
 
-constexpr int kTpRounds = 4;        // exchange rounds of 32 (token, rank) pairs: tile * N <= 128
 constexpr int kTpStages = 3;        // shared-memory stages per warp
 constexpr int kTpMaxCtaWarps = 8;
 constexpr int kTpHeaderWords = 32;  // 256-byte header in front of the slots (64-bit words)
@@ -157,7 +159,7 @@ __device__ __forceinline__ bool tp_poll2(const unsigned long long* sq, const uns
 // issue, shuffles, push, poll); with R tokens side by side that work is done once per tile:
 // one log2(g)-step shuffle tree gives all R scalars, one store instruction pushes 32
 // (token, rank) pairs (pair p*R + r: token r to rank p), one poll loop collects them, N
-// broadcasts per tensor form all R sums.  R * N <= 32 * kTpRounds.
+// broadcasts per tensor form all R sums.  R * N <= 32.
 template <int LOG_G, class IO>
 __global__ void __launch_bounds__(kTpMaxCtaWarps * 32, 2)
 tp_kernel(const __grid_constant__ TpParams P) {
@@ -263,14 +265,27 @@ tp_kernel(const __grid_constant__ TpParams P) {
   const uint32_t gq_u32 = smem0 + (uint32_t)l * 16u * GV;
   const uint32_t gk_u32 = smem0 + (uint32_t)gq_vecs * 16u + (uint32_t)l * 16u * GV;
 
-  // ---- the exchange: pair number (rd * 32 + lane) = p * tile + r carries token r of the tile to and
-  // from rank p; kTpRounds rounds of 32 pairs cover tile * N <= 128 pairs ---------------------------
+  // ---- the exchange: lane p * tile + r carries token r of the tile to and from rank p
+  // (tile * N <= 32, the host chooses the tile so) ----------------------------------------------------
   const int parity = (int)(P.epoch & 1u);
-  const int xr = lane & (tile - 1);         // token of the tile this lane exchanges (the same in every round)
-  const int xp0 = lane >> (5 - LOG_G);    // rank this lane talks to in round 0; round rd: xp0 + rd * g
-  const long long slot_q_out = tp_slot_index(parity, 0, R.rank, P.N, P.cap) + xr;  // in a peer's inbox
-  const long long slot_k_out = tp_slot_index(parity, 1, R.rank, P.N, P.cap) + xr;
-  const int rounds = (tile * P.N + 31) >> 5;
+  const int xr = lane & (tile - 1);       // token of the tile this lane exchanges
+  const int xp = lane >> (5 - LOG_G);     // rank this lane talks to
+  const bool remote = xp < P.N && xp != R.rank;
+  unsigned long long* push_q = nullptr;        // where this rank's scalars go in rank xp's inbox
+  unsigned long long* push_k = nullptr;
+  const unsigned long long* poll_q = nullptr;  // where rank xp's scalars land in this rank's inbox
+  const unsigned long long* poll_k = nullptr;
+  if (remote) {
+    unsigned long long* peer = R.peer_inbox[xp];
+    if (cq) {
+      push_q = peer + tp_slot_index(parity, 0, R.rank, P.N, P.cap) + xr;
+      poll_q = R.inbox + tp_slot_index(parity, 0, xp, P.N, P.cap) + xr;
+    }
+    if (ck) {
+      push_k = peer + tp_slot_index(parity, 1, R.rank, P.N, P.cap) + xr;
+      poll_k = R.inbox + tp_slot_index(parity, 1, xp, P.N, P.cap) + xr;
+    }
+  }
   const unsigned long long tag = (unsigned long long)P.epoch << 32;
 
   const uint32_t sq_lane = (uint32_t)s * (uint32_t)P.q_row_stride + (uint32_t)l * 16u;  // inside a stage
@@ -353,16 +368,8 @@ tp_kernel(const __grid_constant__ TpParams P) {
       mine_q = __shfl_sync(0xffffffffu, pq, xr << LOG_G);
       mine_k = __shfl_sync(0xffffffffu, pk, xr << LOG_G);
       if (t0 + xr < P.T) {  // a short last tile: rows past the end are stale and never published
-#pragma unroll
-        for (int rd = 0; rd < kTpRounds; ++rd) {
-          if (rd >= rounds) break;
-          const int xp = xp0 + (rd << LOG_G);
-          if (xp < P.N && xp != R.rank) {
-            unsigned long long* peer = R.peer_inbox[xp];
-            if (cq) ptx::st_relaxed_sys_u64(peer + slot_q_out + t0, tag | (unsigned long long)__float_as_uint(mine_q));
-            if (ck) ptx::st_relaxed_sys_u64(peer + slot_k_out + t0, tag | (unsigned long long)__float_as_uint(mine_k));
-          }
-        }
+        if (push_q) ptx::st_relaxed_sys_u64(push_q + t0, tag | (unsigned long long)__float_as_uint(mine_q));
+        if (push_k) ptx::st_relaxed_sys_u64(push_k + t0, tag | (unsigned long long)__float_as_uint(mine_k));
       }
       if (t0 + s < P.T && l == 0) {
         if (R.partial_q != nullptr) R.partial_q[t0 + s] = pq;
@@ -374,42 +381,26 @@ tp_kernel(const __grid_constant__ TpParams P) {
       const long long t0 = t_cur - step;
       const long long t = t0 + s;
       const bool live = t < P.T, xlive = t0 + xr < P.T;
-      float inq[kTpRounds], ink[kTpRounds];  // pair (rd, lane): rank xp's scalars of token xr (own for xp == rank)
-      unsigned missing = 0u;
-      int missing_round = 0;
-#pragma unroll
-      for (int rd = 0; rd < kTpRounds; ++rd) {
-        inq[rd] = held_q;
-        ink[rd] = held_k;
-        if (rd >= rounds) continue;
-        const int xp = xp0 + (rd << LOG_G);
-        bool got = true;
-        if (xlive && xp < P.N && xp != R.rank) {
-          const unsigned long long* src_q = cq ? R.inbox + tp_slot_index(parity, 0, xp, P.N, P.cap) + xr + t0 : nullptr;
-          const unsigned long long* src_k = ck ? R.inbox + tp_slot_index(parity, 1, xp, P.N, P.cap) + xr + t0 : nullptr;
-          got = tp_poll2(src_q, src_k, P.epoch, P.wait_ns, status, inq[rd], ink[rd]);
-        }
-        const unsigned m = __ballot_sync(0xffffffffu, !got);
-        if (m != 0u && missing == 0u) {
-          missing = m;
-          missing_round = rd;
-        }
-      }
+      // lane p*tile + r: rank p's scalars of token r (its own for p == rank, nothing for p >= N)
+      float inq = xp < P.N ? held_q : 0.f, ink = xp < P.N ? held_k : 0.f;
+      bool got = true;
+      if (remote && xlive) got = tp_poll2(poll_q ? poll_q + t0 : nullptr, poll_k ? poll_k + t0 : nullptr, P.epoch, P.wait_ns, status, inq, ink);
+      const unsigned missing = __ballot_sync(0xffffffffu, !got);
       if (missing != 0u) {
         const int bad = __ffs((int)missing) - 1;
-        give_up(kTpPeerTimeout, t0 + (bad & (tile - 1)), (bad >> (5 - LOG_G)) + (missing_round << LOG_G), j + 1 < n_tiles, st_next);
+        give_up(kTpPeerTimeout, t0 + (bad & (tile - 1)), bad >> (5 - LOG_G), j + 1 < n_tiles, st_next);
         return;
       }
-      // all N scalars in ascending rank order, the same on every rank
-      float totq = 0.f, totk = 0.f;
+      // S_global: the N scalars of a token added pairwise over the rank index (ranks 2i and 2i+1,
+      // then pairs of pairs, ...).  Every rank runs the same tree on the same N values, so all ranks
+      // get the same bits; log2 steps instead of N.
 #pragma unroll
-      for (int rd = 0; rd < kTpRounds; ++rd) {
-        for (int pp = 0; pp < g; ++pp) {  // rank rd * g + pp sits in lane pp * tile + s of round rd
-          if ((rd << LOG_G) + pp >= P.N) break;
-          totq += __shfl_sync(0xffffffffu, inq[rd], pp * tile + s);
-          totk += __shfl_sync(0xffffffffu, ink[rd], pp * tile + s);
-        }
+      for (int o = tile; o < 32; o <<= 1) {
+        inq += __shfl_xor_sync(0xffffffffu, inq, o);
+        ink += __shfl_xor_sync(0xffffffffu, ink, o);
       }
+      const float totq = __shfl_sync(0xffffffffu, inq, s);  // lane s = (rank 0, token s) holds token s's sum
+      const float totk = __shfl_sync(0xffffffffu, ink, s);
       const float rq = rstd_of(totq, P.inv_dq, P.eps);
       const float rk = rstd_of(totk, P.inv_dk, P.eps);
       if (live) {

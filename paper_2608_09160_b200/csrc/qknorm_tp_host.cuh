@@ -129,7 +129,7 @@ int run_tp(int elem_bytes, const qknorm_tp_rank* ranks, int n_local, int N, long
   int log_g = 5;
   for (int lg = 2; lg <= 5; ++lg) {
     const int tile = 32 >> lg;
-    if (tile * N > 32 * kTpRounds) continue;
+    if (tile * N > 32) continue;  // one lane per (token, rank) pair
     if (forced_log_g >= 0 ? lg != forced_log_g : (tile > 1 && tile * row_bytes > tile_bytes_max)) continue;
     log_g = lg;
     break;

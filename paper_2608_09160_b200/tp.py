@@ -7,7 +7,7 @@ the library's kernel.
 Two ways to use it:
 
 * ``EmulatedGroup`` -- all N ranks' buffers on ONE GPU, one cooperative launch serves
-  them all.  The protocol (push, tagged slots, bounded polls, rank-order sum) is the real
+  them all.  The protocol (push, tagged slots, bounded polls, one fixed sum order) is the real
   one; only the "link" is the GPU's own memory.  Tests and the benchmark use this.
 * ``Communicator`` -- one process per GPU over ``torch.distributed``: each rank creates
   its inbox, the inter-process handles are all-gathered on the host, and every call

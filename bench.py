@@ -312,27 +312,26 @@ def config_table(steps: int, warmup: int, peak: float, skip: str):
     todo += [(name, W.WORKLOADS[name].shards[-1], "e4m3") for name in ("C3", "C4", "C5")]
     for name, S, io in todo:
         w = W.WORKLOADS[name]
-        if True:
-            key = f"{name}/S{S}" + ("" if io == "bf16" else "/e4m3")
-            if key == skip:
-                continue
-            case = DeviceCase(w, S, io=io)
-            ts = time_calls(case.call, max(steps, 10), max(warmup, 3))
-            med, mn = statistics.median(ts), min(ts)
-            row = {"us_median": round(med * 1e3, 3), "us_min": round(mn * 1e3, 3),
-                   "GBps": round(case.bytes / (med * 1e-3) / 1e9, 1),
-                   "frac_measured_peak": round(case.bytes / (med * 1e-3) / 1e9 / peak, 4),
-                   "frac_nominal_8TBps": round(case.bytes / (med * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
-                   "bytes": case.bytes, "variant": binding.last_variant(),
-                   "l2": "resident (working set < L2)" if case.bytes < 100e6 else "inputs larger than L2",
-                   "same_size_copy_GBps": None}
-            if w.tokens <= 1024:
-                row["us_graph_replay"] = round(graph_replay_us(case), 3)
-            else:
-                row["same_size_copy_GBps"] = round(copy_rate_same_bytes(case.bytes), 1)
-            rows[key] = row
-            del case
-            torch.cuda.empty_cache()
+        key = f"{name}/S{S}" + ("" if io == "bf16" else "/e4m3")
+        if key == skip:
+            continue
+        case = DeviceCase(w, S, io=io)
+        ts = time_calls(case.call, max(steps, 10), max(warmup, 3))
+        med, mn = statistics.median(ts), min(ts)
+        row = {"us_median": round(med * 1e3, 3), "us_min": round(mn * 1e3, 3),
+               "GBps": round(case.bytes / (med * 1e-3) / 1e9, 1),
+               "frac_measured_peak": round(case.bytes / (med * 1e-3) / 1e9 / peak, 4),
+               "frac_nominal_8TBps": round(case.bytes / (med * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
+               "bytes": case.bytes, "variant": binding.last_variant(),
+               "l2": "resident (working set < L2)" if case.bytes < 100e6 else "inputs larger than L2",
+               "same_size_copy_GBps": None}
+        if w.tokens <= 1024:
+            row["us_graph_replay"] = round(graph_replay_us(case), 3)
+        else:
+            row["same_size_copy_GBps"] = round(copy_rate_same_bytes(case.bytes), 1)
+        rows[key] = row
+        del case
+        torch.cuda.empty_cache()
     rows.update(variant_rows(steps, warmup, peak))
     rows.update(baseline_rows(steps, warmup, peak))
     rows.update(tp_rows(steps, warmup, peak))

@@ -47,6 +47,7 @@ from paper_2608_09160_b200 import workloads as W  # noqa: E402
 METRIC = "qknorm_prefill_GBps"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
+L2_BYTES = 126e6          # B200 L2 capacity
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes (read + write) per launch of the dominant kernel measured by ncu
@@ -292,6 +293,43 @@ def graph_replay_us(case: DeviceCase, calls_per_graph: int = 50, replays: int = 
     return statistics.median(ts)
 
 
+def graph_replay_cold_us(case: DeviceCase, replays: int = 10) -> float:
+    """us per call with the call's data NOT in L2: one CUDA graph of K calls, each on its own copy of
+    the buffers, K chosen so that the copies together are more than twice the 126 MB L2; by the time a
+    replay comes back to a copy, everything the graph touched since has pushed it out."""
+    sets = max(4, int(2.2 * L2_BYTES / max(case.bytes, 1)) + 1)
+    dev = case.dev
+
+    def clones(ts):
+        return [[t.clone() for t in ts] for _ in range(sets)]
+    qs, ks = clones(dev["q"]), clones(dev["k"])
+    oqs = qs if case.w.in_place else clones(dev["q"])
+    oks = ks if case.w.in_place else clones(dev["k"])
+    calls = [case._prepared(qs[i], ks[i], oqs[i], oks[i]) for i in range(sets)]
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        calls[0]()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for c in calls:
+            c()
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(replays):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b) * 1e3 / sets)
+    return statistics.median(ts)
+
+
 def copy_rate_same_bytes(nbytes: int, steps: int = 10) -> float:
     """GB/s (read + write bytes) of a device-to-device copy that moves the same number of
     bytes as one call: what a plain memcpy of this size reaches on this GPU, ramp-up included."""
@@ -326,7 +364,8 @@ def config_table(steps: int, warmup: int, peak: float, skip: str):
                "l2": "resident (working set < L2)" if case.bytes < 100e6 else "inputs larger than L2",
                "same_size_copy_GBps": None}
         if w.tokens <= 1024:
-            row["us_graph_replay"] = round(graph_replay_us(case), 3)
+            row["us_graph_replay"] = round(graph_replay_us(case), 3)            # L2-warm, launch amortised
+            row["us_graph_replay_l2_cold"] = round(graph_replay_cold_us(case), 3)  # every call on data not in L2
         else:
             row["same_size_copy_GBps"] = round(copy_rate_same_bytes(case.bytes), 1)
         rows[key] = row
@@ -468,10 +507,16 @@ def cpu_baseline(w: W.Workload, target_cpu_seconds: float = 16.0):
     ws, bits = oracle_sample_inputs(w, n)
     dt = run_oracle_once(bits, w.eps, cores)
     gbs = ws.algorithmic_bytes / dt / 1e9
+    # the same oracle on ONE thread, on a sample 1/cores as long (about a second)
+    n1 = max(64, n // max(cores, 1))
+    ws1, bits1 = oracle_sample_inputs(w, n1)
+    dt1 = run_oracle_once(bits1, w.eps, 1)
     return {"value": round(gbs, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {n} of {w.tokens} tokens of {w.name} (dq={w.dq}, dk={w.dk}), "
                       f"unsharded definition, one pass, {dt:.2f} s wall",
-            "seconds": round(dt, 3)}
+            "seconds": round(dt, 3),
+            "single_thread": {"value": round(ws1.algorithmic_bytes / dt1 / 1e9, 4), "unit": UNIT, "cores": 1,
+                              "sample": f"first {n1} tokens, one pass, {dt1:.2f} s wall"}}
 
 
 def rank_workload(w: W.Workload, rank: int) -> W.Workload:

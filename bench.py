@@ -615,6 +615,7 @@ def main():
                     help="only the tensor-parallel rows of the table (all ranks on this GPU), as one JSON object; "
                          "with --tokens for a small case to profile")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-chunks", type=int, default=8, help="token chunks of the host-to-host pipeline")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -682,7 +683,7 @@ def main():
     # ---- end to end: host buffers in, host buffers out ----------------------------------------
     e2e = None
     if not args.no_e2e:
-        e2e_chunks = case.prepare_e2e()
+        e2e_chunks = case.prepare_e2e(args.e2e_chunks)
         for _ in range(2):
             case.e2e_step()
         barrier()

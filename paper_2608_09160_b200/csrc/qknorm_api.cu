@@ -15,6 +15,8 @@
 #include "qknorm_params.h"
 #include "qknorm_ring.cuh"
 #include "qknorm_rows.cuh"
+#include "../../include/qknorm_tp.h"
+#include "qknorm_tp.cuh"
 #include "qknorm_warp.cuh"
 
 namespace qknorm {
@@ -73,7 +75,7 @@ WarpKernel warp_kernel_for(int l, bool exact, int elem_bytes) {
 }
 
 // Set by a ring kernel whose bounded wait ran out (0 = never happened).
-__device__ int g_ring_error = 0;
+__device__ __align__(8) int g_ring_error[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // word 0 is the error word; 1-2: where it happened
 
 // Built-in scratch of qknorm_baseline_two_pass_static: 1 MiB of device memory that every
 // GPU which loads this library holds until the process exits.  In host code this name is
@@ -344,6 +346,8 @@ int finish_launch(const char* variant) {
   return QKNORM_OK;
 }
 
+#include "qknorm_tp_host.cuh"  // run_tp, launch_tile
+
 // The TMA ring kernel (prefill sizes).  Returns QKNORM_OK with *done = false when
 // the shape does not fit it and another variant should run.
 int launch_ring(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* done) {
@@ -475,6 +479,12 @@ int launch(Params& P, cudaStream_t stream) {
 
   if (!force_general && vector_path_ok(P)) {
     const bool latency = P.T < 4LL * sms;
+    const bool force_warp = force && strcmp(force, "warp") == 0;
+    if (!latency && !force_rows && !force_ring && !force_warp) {
+      bool done = false;
+      rc = launch_tile(P, *dev, stream, &done);  // short unsharded rows: several tokens per warp
+      if (rc != QKNORM_OK || done) return rc;
+    }
     if (!latency && !force_rows && !force_ring) {
       bool done = false;
       rc = launch_warp(P, *dev, stream, &done);
@@ -777,7 +787,7 @@ int static_scratch_address(float** out) {
 }  // namespace
 }  // namespace qknorm
 
-#include "qknorm_tp_host.cuh"  // the tensor-parallel entry points (include/qknorm_tp.h)
+#include "qknorm_tp_abi.cuh"  // the tensor-parallel entry points (include/qknorm_tp.h)
 
 extern "C" {
 

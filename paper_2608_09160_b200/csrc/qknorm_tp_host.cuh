@@ -1,20 +1,78 @@
-// Host side of the tensor-parallel entry points (include/qknorm_tp.h): validation,
-// grid choice and the cooperative launch of tp_kernel, plus the inbox helpers.
-// Included by qknorm_api.cu after its own helpers (device cache, occupancy cache,
-// overlap test), which it uses.
+// Host side of the tiled kernel (qknorm_tp.cuh): validation, tile and grid choice, launch --
+// cooperative for the tensor-parallel entry points of include/qknorm_tp.h, plain for the narrow
+// unsharded rows the main entry points hand to the same kernel.
+// Included by qknorm_api.cu INSIDE its unnamed namespace, after the helpers it uses (device cache,
+// occupancy cache, overlap test).
 #pragma once
-#include "../../include/qknorm_tp.h"
-#include "qknorm_tp.cuh"
-
-namespace qknorm {
-
-namespace {
 
 int tp_inbox_bytes(int num_ranks, long long cap, long long* bytes) {
   if (!bytes) return QKNORM_ERR_NULL;
   if (num_ranks < 1 || num_ranks > kMaxShards) return QKNORM_ERR_SHARDS;
   if (cap < 1 || cap > (1LL << 31)) return QKNORM_ERR_SHAPE;
   *bytes = 8LL * (kTpHeaderWords + 4LL * num_ranks * cap);
+  return QKNORM_OK;
+}
+
+// Tile shape, stage layout, CTA size and kernel for the slice widths in P (wq, wk, N already set).
+// Host arithmetic only; QKNORM_ERR_SHAPE when a slice row pair is too long for the kernel.
+int tp_configure(TpParams& P, int elem_bytes, int* warps_out, int* smem_out, TpKernel* fn_out) {
+  const int wq = P.wq, wk = P.wk, N = P.N;
+  // Tokens per warp tile: R = 32 / g lane groups of g lanes, one token each.  More tokens per tile
+  // spread the per-tile work (barrier waits, copy issue, shuffles, push, poll) over more rows; the
+  // tile's bytes times the three stages times the warps must fit the SM's shared memory.  Measured
+  // on B200 (8 ranks on one GPU): tiles of 9-12 KB are fastest, 5 KB and 18 KB both cost 15-30 %.
+  const int cq = wq * elem_bytes / 16, ck = wk * elem_bytes / 16;
+  const int row_bytes = (wq + wk) * elem_bytes;
+  const int tile_bytes_max = env_int("QKNORM_TP_TILE_BYTES", 12000);
+  const int forced_log_g = env_int("QKNORM_TP_LOG_G", -1);
+  int log_g = 5;
+  for (int lg = 2; lg <= 5; ++lg) {
+    const int tile = 32 >> lg;
+    if (tile * N > 32) continue;  // one lane per (token, rank) pair
+    if (forced_log_g >= 0 ? lg != forced_log_g : (tile > 1 && tile * row_bytes > tile_bytes_max)) continue;
+    log_g = lg;
+    break;
+  }
+  TpKernel fn = tp_kernel_for(log_g, elem_bytes);
+  if (!fn) return QKNORM_ERR_SHAPE;
+  const int tile = 32 >> log_g;
+  {
+    const int g = 1 << log_g;
+    P.log_g = log_g;
+    // rows of a tile side by side in the stage; the skew keeps lane groups that read in the same
+    // quarter-warp on different banks
+    const int skew = (tile > 1 && g < 8) ? g * 16 : 0;
+    P.q_row_stride = cq ? wq * elem_bytes + skew : 0;
+    P.k_row_stride = ck ? wk * elem_bytes + skew : 0;
+    P.k_base = tile * P.q_row_stride;
+    P.stage_bytes = round_up(P.k_base + tile * P.k_row_stride, 128);
+    P.gamma_bytes = round_up((wq + wk) * 2, 128);
+  }
+
+  // Warps per CTA: the CTA size that puts the most warps on an SM (three stages per warp and one
+  // copy of gamma per CTA against the SM's shared memory; 128 registers per thread allow 16 warps);
+  // among equals the larger CTA, which shares gamma between more warps.
+  constexpr int kSmemPerCta = 227 * 1024;  // sm_100: opt-in maximum of dynamic shared memory per CTA
+  constexpr int kSmemPerSm = 228 * 1024;   // and what one SM has, of which every resident CTA reserves 1 KB
+  const int forced_warps = env_int("QKNORM_TP_WARPS", 0);
+  int warps = 0, best_per_sm = 0;
+  for (int w = kTpMaxCtaWarps; w >= 1; --w) {
+    if (forced_warps > 0 && w != forced_warps) continue;
+    const int bytes = P.gamma_bytes + w * kTpStages * P.stage_bytes;
+    if (bytes > kSmemPerCta) continue;
+    int per_sm = (kSmemPerSm / (bytes + 1024 + 256)) * w;
+    if (per_sm > 16) per_sm = 16;
+    if (per_sm > best_per_sm) {
+      best_per_sm = per_sm;
+      warps = w;
+    }
+  }
+  if (warps == 0) return QKNORM_ERR_SHAPE;  // a slice row pair too long for three stages of shared memory
+  const int smem = P.gamma_bytes + warps * kTpStages * P.stage_bytes;
+
+  *warps_out = warps;
+  *smem_out = smem;
+  *fn_out = fn;
   return QKNORM_OK;
 }
 
@@ -118,58 +176,11 @@ int run_tp(int elem_bytes, const qknorm_tp_rank* ranks, int n_local, int N, long
       if (may_overlap(outs[i], others[j])) return QKNORM_ERR_ALIAS;
   }
 
-  // Tokens per warp tile: R = 32 / g lane groups of g lanes, one token each.  More tokens per tile
-  // spread the per-tile work (barrier waits, copy issue, shuffles, push, poll) over more rows; the
-  // tile's bytes times the three stages times the warps must fit the SM's shared memory.  Measured
-  // on B200 (8 ranks on one GPU): tiles of 9-12 KB are fastest, 5 KB and 18 KB both cost 15-30 %.
-  const int cq = wq * elem_bytes / 16, ck = wk * elem_bytes / 16;
-  const int row_bytes = (wq + wk) * elem_bytes;
-  const int tile_bytes_max = env_int("QKNORM_TP_TILE_BYTES", 12000);
-  const int forced_log_g = env_int("QKNORM_TP_LOG_G", -1);
-  int log_g = 5;
-  for (int lg = 2; lg <= 5; ++lg) {
-    const int tile = 32 >> lg;
-    if (tile * N > 32) continue;  // one lane per (token, rank) pair
-    if (forced_log_g >= 0 ? lg != forced_log_g : (tile > 1 && tile * row_bytes > tile_bytes_max)) continue;
-    log_g = lg;
-    break;
-  }
-  TpKernel fn = tp_kernel_for(log_g, elem_bytes);
-  if (!fn) return QKNORM_ERR_SHAPE;
-  const int tile = 32 >> log_g;
-  {
-    const int g = 1 << log_g;
-    P.log_g = log_g;
-    // rows of a tile side by side in the stage; the skew keeps lane groups that read in the same
-    // quarter-warp on different banks
-    const int skew = (tile > 1 && g < 8) ? g * 16 : 0;
-    P.q_row_stride = cq ? wq * elem_bytes + skew : 0;
-    P.k_row_stride = ck ? wk * elem_bytes + skew : 0;
-    P.k_base = tile * P.q_row_stride;
-    P.stage_bytes = round_up(P.k_base + tile * P.k_row_stride, 128);
-    P.gamma_bytes = round_up((wq + wk) * 2, 128);
-  }
-
-  // Warps per CTA: the CTA size that puts the most warps on an SM (three stages per warp and one
-  // copy of gamma per CTA against the SM's shared memory; 128 registers per thread allow 16 warps);
-  // among equals the larger CTA, which shares gamma between more warps.
-  constexpr int kSmemPerCta = 227 * 1024;  // sm_100: opt-in maximum of dynamic shared memory per CTA
-  constexpr int kSmemPerSm = 228 * 1024;   // and what one SM has, of which every resident CTA reserves 1 KB
-  const int forced_warps = env_int("QKNORM_TP_WARPS", 0);
-  int warps = 0, best_per_sm = 0;
-  for (int w = kTpMaxCtaWarps; w >= 1; --w) {
-    if (forced_warps > 0 && w != forced_warps) continue;
-    const int bytes = P.gamma_bytes + w * kTpStages * P.stage_bytes;
-    if (bytes > kSmemPerCta) continue;
-    int per_sm = (kSmemPerSm / (bytes + 1024 + 256)) * w;
-    if (per_sm > 16) per_sm = 16;
-    if (per_sm > best_per_sm) {
-      best_per_sm = per_sm;
-      warps = w;
-    }
-  }
-  if (warps == 0) return QKNORM_ERR_SHAPE;  // a slice row pair too long for three stages of shared memory
-  const int smem = P.gamma_bytes + warps * kTpStages * P.stage_bytes;
+  int warps = 0, smem = 0;
+  TpKernel fn = nullptr;
+  rc = tp_configure(P, elem_bytes, &warps, &smem, &fn);
+  if (rc != QKNORM_OK) return rc;
+  const int tile = 32 >> P.log_g;
 
   const DeviceInfo* dev = nullptr;
   rc = current_device(&dev);
@@ -195,107 +206,67 @@ int run_tp(int elem_bytes, const qknorm_tp_rank* ranks, int n_local, int N, long
   return finish_launch("tp");
 }
 
-}  // namespace
-}  // namespace qknorm
 
-extern "C" {
 
-int qknorm_tp_inbox_bytes(int32_t num_ranks, int64_t token_capacity, int64_t* bytes) {
-  long long b = 0;
-  const int rc = qknorm::tp_inbox_bytes(num_ranks, token_capacity, bytes ? &b : nullptr);
-  if (rc == QKNORM_OK) *bytes = b;
+// Unsharded rows too short for one token per warp (a few KB): the tiled kernel with a single rank
+// and therefore no exchange -- several tokens side by side per warp, three stages per warp.
+// Measured on B200, 600 MB of rows: at 640-byte rows the warp-per-token kernel reaches 1.5 TB/s
+// and this one 5.5 TB/s; they meet near 2.8 KB (bf16) and 4 KB (FP8-E4M3), above which the
+// warp-per-token kernel is 5-8 % faster.  Returns QKNORM_OK with *done = false when the call is
+// not of that kind.
+int launch_tile(const Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* done) {
+  *done = false;
+  if (P.S != 1) return QKNORM_OK;
+  const int row_bytes = (P.q.d + P.k.d) * P.elem_bytes;
+  const int limit = env_int("QKNORM_TILE_MAX_ROW_BYTES", P.elem_bytes == 1 ? 4096 : 2816);
+  if (row_bytes > limit) return QKNORM_OK;
+  TpParams T;
+  memset(&T, 0, sizeof(T));
+  T.n_local = 1;
+  T.N = 1;
+  T.T = P.T;
+  T.cap = P.T;
+  T.wq = P.q.d;
+  T.wk = P.k.d;
+  T.ldxq = P.q.ldx;
+  T.ldxk = P.k.ldx;
+  T.ldyq = P.q.ldy;
+  T.ldyk = P.k.ldy;
+  T.inv_dq = P.q.inv_d;
+  T.inv_dk = P.k.inv_d;
+  T.eps = P.eps;
+  T.epoch = 1u;  // no peer, nothing is ever polled
+  T.wait_ns = 1000000000ull;
+  TpRank& r = T.r[0];
+  r.rank = 0;
+  r.xq = P.q.x[0];
+  r.xk = P.k.x[0];
+  r.gq = P.q.gamma[0];
+  r.gk = P.k.gamma[0];
+  r.yq = P.q.y[0];
+  r.yk = P.k.y[0];
+  r.rstd_q = P.q.rstd;
+  r.rstd_k = P.k.rstd;
+  r.partial_q = P.q.partials;  // with one slice the slice's scalar is the row's
+  r.partial_k = P.k.partials;
+  r.inbox = reinterpret_cast<unsigned long long*>(dev.ring_error);  // only its status words are used
+  int warps = 0, smem = 0;
+  TpKernel fn = nullptr;
+  int rc = tp_configure(T, P.elem_bytes, &warps, &smem, &fn);
+  if (rc != QKNORM_OK) return QKNORM_OK;  // does not fit: another variant takes the call
+  if (smem > dev.smem_per_block) return QKNORM_OK;
+  rc = allow_dynamic_smem((const void*)fn, smem);
+  if (rc != QKNORM_OK) return rc;
+  int resident = 1;
+  rc = resident_blocks((const void*)fn, warps * 32, smem, &resident);
+  if (rc != QKNORM_OK) return rc;
+  const int tile = 32 >> T.log_g;
+  const long long tiles = (P.T + tile - 1) / tile;
+  const long long needed = (tiles + warps - 1) / warps;
+  long long grid = (long long)resident * dev.sm_count;  // bounded grid of co-resident CTAs
+  if (grid > needed) grid = needed;
+  fn<<<(unsigned)grid, warps * 32, smem, stream>>>(T);
+  rc = finish_launch("tile");
+  *done = rc == QKNORM_OK;
   return rc;
 }
-
-int qknorm_fwd_tp(const qknorm_tp_rank* ranks, int32_t n_local, int32_t num_ranks, int64_t tokens,
-                  int64_t token_capacity, int32_t wq, int32_t wk, const int64_t* ld, float eps, uint32_t epoch,
-                  uint32_t wait_limit_us, void* stream) {
-  return qknorm::run_tp(2, ranks, n_local, num_ranks, tokens, token_capacity, wq, wk, ld, eps, epoch,
-                        wait_limit_us, (cudaStream_t)stream);
-}
-
-int qknorm_fwd_tp_e4m3(const qknorm_tp_rank* ranks, int32_t n_local, int32_t num_ranks, int64_t tokens,
-                       int64_t token_capacity, int32_t wq, int32_t wk, const int64_t* ld, float eps, uint32_t epoch,
-                       uint32_t wait_limit_us, void* stream) {
-  return qknorm::run_tp(1, ranks, n_local, num_ranks, tokens, token_capacity, wq, wk, ld, eps, epoch,
-                        wait_limit_us, (cudaStream_t)stream);
-}
-
-int qknorm_tp_status(const void* inbox, int32_t* out) {
-  if (!inbox || !out) return QKNORM_ERR_NULL;
-  cudaError_t e = cudaMemcpy(out, inbox, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost);
-  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
-  return QKNORM_OK;
-}
-
-int qknorm_tp_clear_status(void* inbox, void* stream) {
-  if (!inbox) return QKNORM_ERR_NULL;
-  cudaError_t e = cudaMemsetAsync(inbox, 0, 8 * qknorm::kTpHeaderWords, (cudaStream_t)stream);
-  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
-  return QKNORM_OK;
-}
-
-int qknorm_tp_inbox_create(int32_t num_ranks, int64_t token_capacity, void** out) {
-  if (!out) return QKNORM_ERR_NULL;
-  long long bytes = 0;
-  const int rc = qknorm::tp_inbox_bytes(num_ranks, token_capacity, &bytes);
-  if (rc != QKNORM_OK) return rc;
-  void* p = nullptr;
-  cudaError_t e = cudaMalloc(&p, (size_t)bytes);
-  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
-  e = cudaMemset(p, 0, (size_t)bytes);
-  if (e == cudaSuccess) e = cudaDeviceSynchronize();
-  if (e != cudaSuccess) {
-    cudaFree(p);
-    return qknorm::set_cuda_error(e);
-  }
-  *out = p;
-  return QKNORM_OK;
-}
-
-int qknorm_tp_inbox_zero(void* inbox, int32_t num_ranks, int64_t token_capacity, void* stream) {
-  if (!inbox) return QKNORM_ERR_NULL;
-  long long bytes = 0;
-  const int rc = qknorm::tp_inbox_bytes(num_ranks, token_capacity, &bytes);
-  if (rc != QKNORM_OK) return rc;
-  cudaError_t e = cudaMemsetAsync(inbox, 0, (size_t)bytes, (cudaStream_t)stream);
-  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
-  return QKNORM_OK;
-}
-
-int qknorm_tp_inbox_destroy(void* inbox) {
-  if (!inbox) return QKNORM_OK;
-  cudaError_t e = cudaFree(inbox);
-  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
-  return QKNORM_OK;
-}
-
-int qknorm_tp_ipc_export(const void* inbox, unsigned char* handle) {
-  static_assert(sizeof(cudaIpcMemHandle_t) == QKNORM_TP_IPC_HANDLE_BYTES, "handle size");
-  if (!inbox || !handle) return QKNORM_ERR_NULL;
-  cudaIpcMemHandle_t h;
-  cudaError_t e = cudaIpcGetMemHandle(&h, const_cast<void*>(inbox));
-  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
-  memcpy(handle, &h, sizeof(h));
-  return QKNORM_OK;
-}
-
-int qknorm_tp_ipc_open(const unsigned char* handle, void** out) {
-  if (!handle || !out) return QKNORM_ERR_NULL;
-  cudaIpcMemHandle_t h;
-  memcpy(&h, handle, sizeof(h));
-  void* p = nullptr;
-  cudaError_t e = cudaIpcOpenMemHandle(&p, h, cudaIpcMemLazyEnablePeerAccess);
-  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
-  *out = p;
-  return QKNORM_OK;
-}
-
-int qknorm_tp_ipc_close(void* mapped) {
-  if (!mapped) return QKNORM_OK;
-  cudaError_t e = cudaIpcCloseMemHandle(mapped);
-  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
-  return QKNORM_OK;
-}
-
-}  // extern "C"

@@ -186,6 +186,10 @@ def small_parity_shapes() -> List[Workload]:
         ("s_prefill_s16", 640, 4096, 1024, (16,)),       # two lanes per shard, every lane issues a bulk copy
         ("s_prefill_s5", 610, 2240, 560, (5, 7)),        # shard counts that are not powers of two
         ("s_prefill_wide", 600, 16384, 4096, (1, 4)),    # rows too wide for one warp: the CTA-per-token TMA ring
+        ("s_tile_gqa", 3001, 1024, 128, (1,)),           # short unsharded rows: several tokens per warp, ragged last tile
+        ("s_tile_tiny", 1000, 64, 8, (1,)),              # 128-byte and 16-byte rows
+        ("s_tile_konly", 777, 0, 256, (1,)),
+        ("s_tile_qonly", 601, 1280, 0, (1,)),
     ]
     out = []
     for i, (name, t, dq, dk, sh) in enumerate(shapes):

@@ -22,7 +22,7 @@ SHAPES = [
     ("e_gqa", 900, 5120, 1024, (8, 1), ("warp", "warp")),
     ("e_mha", 700, 5120, 5120, (4,), ("warp",)),
     ("e_odd_width", 650, 1000, 136, (1,), ("general",)),          # not a multiple of 16 elements
-    ("e_ragged", 777, 1008, 144, (1, 3), ("warp", "warp")),       # multiples of 16, ragged over the lanes
+    ("e_ragged", 777, 1008, 144, (1, 3), ("tile", "warp")),       # multiples of 16, ragged over the lanes
     ("e_tiny", 3, 16, 16, (1,), ("rows",)),
     ("e_konly", 600, 0, 2048, (2,), ("warp",)),
 ]
@@ -128,10 +128,11 @@ def test_full_size_e4m3(libqknorm, name):
         print(f"{name} e4m3 {nm}: rate at distance 1 {rate:.2e}")
 
 
-def test_e4m3_gamma_outside_fp16_takes_the_bf16_gamma_path(libqknorm):
-    """The prefill kernel keeps an fp16 copy of gamma when every value fits fp16; one value that
+@pytest.mark.parametrize("dq,dk,variant", [(2048, 512, "tile"), (8192, 1024, "warp")])
+def test_e4m3_gamma_outside_fp16_takes_the_bf16_gamma_path(libqknorm, dq, dk, variant):
+    """The prefill kernels keep an fp16 copy of gamma when every value fits fp16; one value that
     does not (2^-20, 1e5) must switch the whole call to the bf16-gamma arithmetic with the same result."""
-    w = W.Workload("e_wide_gamma", tokens=700, dq=2048, dk=512, shards=(1,), seed=31, sigma=1.5)
+    w = W.Workload("e_wide_gamma", tokens=700, dq=dq, dk=dk, shards=(1,), seed=31, sigma=1.5)
     inp = W.make_inputs_e4m3(w)
     gq = inp["gamma_q"].clone()
     gq[5] = 2.0 ** -20
@@ -141,7 +142,7 @@ def test_e4m3_gamma_outside_fp16_takes_the_bf16_gamma_path(libqknorm):
     ref_k = oracle.rmsnorm_e4m3([W.e4m3_bits(inp["k"])], [W.bf16_bits(inp["gamma_k"])], w.eps)["y"][0]
     oq, ok = binding.qknorm_fwd_e4m3(inp["q"].cuda(), inp["k"].cuda(), gq.cuda(), inp["gamma_k"].cuda(), w.eps)
     torch.cuda.synchronize()
-    assert binding.last_variant() == "warp"
+    assert binding.last_variant() == variant
     compare_e4m3(W.e4m3_bits(oq.cpu()), ref_q, "wide gamma q")
     compare_e4m3(W.e4m3_bits(ok.cpu()), ref_k, "wide gamma k")
     assert (W.e4m3_bits(oq.cpu())[:, 77] & 0x7F == 0x7E).mean() > 0.5     # 1e5 * x saturates

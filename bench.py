@@ -473,6 +473,20 @@ def variant_rows(steps: int, warmup: int, peak: float):
                          "bytes": w.algorithmic_bytes, "variant": binding.last_variant(), "l2": "inputs larger than L2"}
         del buf, q, k
         torch.cuda.empty_cache()
+    # short rows: what ONE of 8 tensor-parallel ranks holds of C5 (its column slice), normalised on
+    # its own as unsharded rows -- the shape the tiled kernel exists for
+    w = W.Workload("C5-slice", tokens=65536, dq=1024, dk=128, shards=(1,), sigma=2.0, seed=4, in_place=True)
+    case = DeviceCase(w, 1)
+    ts = time_calls(case.call, max(steps, 10), max(warmup, 3))
+    med = statistics.median(ts)
+    gbs = case.bytes / (med * 1e-3) / 1e9
+    rows["C5-one-rank-slice(1024+128)/unsharded/in-place"] = {
+        "us_median": round(med * 1e3, 3), "us_min": round(min(ts) * 1e3, 3), "GBps": round(gbs, 1),
+        "frac_measured_peak": round(gbs / peak, 4), "frac_nominal_8TBps": round(gbs / NOMINAL_HBM_GBS, 4),
+        "bytes": case.bytes, "variant": binding.last_variant(), "l2": "inputs larger than L2",
+        "same_size_copy_GBps": round(copy_rate_same_bytes(case.bytes), 1)}
+    del case
+    torch.cuda.empty_cache()
     return rows
 
 

@@ -478,8 +478,21 @@ int launch(Params& P, cudaStream_t stream) {
   const bool force_ring = force && strcmp(force, "ring") == 0;
 
   if (!force_general && vector_path_ok(P)) {
-    const bool latency = P.T < 4LL * sms;
     const bool force_warp = force && strcmp(force, "warp") == 0;
+    const bool force_tile = force && strcmp(force, "tile") == 0;
+    // Which regime: the register-resident rows kernel (a CTA per token, nothing staged, no set-up
+    // beyond gamma in registers) finishes a call of a thousand or two tokens in fewer microseconds
+    // than the TMA-fed kernels need to get going.  Measured on B200 over row widths of 1 to 32 KB and
+    // 1 to 16 slices, from L2 and from HBM: the crossover sits between 1000 and 2900 tokens, earlier
+    // when the slices are many and narrow (CTAs of more than 384 threads).
+    bool latency = P.T < 4LL * sms;
+    if (!latency && !force_warp && !force_ring && !force_tile) {
+      RowsPlan plan;
+      if (plan_rows(P, /*latency=*/true, &plan)) {
+        const long long most = env_int("QKNORM_ROWS_MAX_TOKENS", plan.threads <= 384 ? 2048 : 1280);
+        if (P.T <= most) latency = true;
+      }
+    }
     if (!latency && !force_rows && !force_ring && !force_warp) {
       bool done = false;
       rc = launch_tile(P, *dev, stream, &done);  // short unsharded rows: several tokens per warp

@@ -15,7 +15,8 @@ int tp_inbox_bytes(int num_ranks, long long cap, long long* bytes) {
 
 // Tile shape, stage layout, CTA size and kernel for the slice widths in P (wq, wk, N already set).
 // Host arithmetic only; QKNORM_ERR_SHAPE when a slice row pair is too long for the kernel.
-int tp_configure(TpParams& P, int elem_bytes, int* warps_out, int* smem_out, TpKernel* fn_out) {
+// `sm_count` (0 = unknown) lets short calls take smaller CTAs so that every SM gets one.
+int tp_configure(TpParams& P, int elem_bytes, int sm_count, int* warps_out, int* smem_out, TpKernel* fn_out) {
   const int wq = P.wq, wk = P.wk, N = P.N;
   // Tokens per warp tile: R = 32 / g lane groups of g lanes, one token each.  More tokens per tile
   // spread the per-tile work (barrier waits, copy issue, shuffles, push, poll) over more rows; the
@@ -55,8 +56,14 @@ int tp_configure(TpParams& P, int elem_bytes, int* warps_out, int* smem_out, TpK
   constexpr int kSmemPerCta = 227 * 1024;  // sm_100: opt-in maximum of dynamic shared memory per CTA
   constexpr int kSmemPerSm = 228 * 1024;   // and what one SM has, of which every resident CTA reserves 1 KB
   const int forced_warps = env_int("QKNORM_TP_WARPS", 0);
+  int max_warps = kTpMaxCtaWarps;
+  if (sm_count > 0) {  // few tiles: no more warps per CTA than leaves a CTA for every SM (and every local rank)
+    const long long tiles = (P.T + tile - 1) / tile;
+    const long long fair = (tiles * P.n_local + sm_count - 1) / sm_count;
+    if (fair < max_warps) max_warps = fair < 1 ? 1 : (int)fair;
+  }
   int warps = 0, best_per_sm = 0;
-  for (int w = kTpMaxCtaWarps; w >= 1; --w) {
+  for (int w = max_warps; w >= 1; --w) {
     if (forced_warps > 0 && w != forced_warps) continue;
     const int bytes = P.gamma_bytes + w * kTpStages * P.stage_bytes;
     if (bytes > kSmemPerCta) continue;
@@ -178,12 +185,14 @@ int run_tp(int elem_bytes, const qknorm_tp_rank* ranks, int n_local, int N, long
 
   int warps = 0, smem = 0;
   TpKernel fn = nullptr;
-  rc = tp_configure(P, elem_bytes, &warps, &smem, &fn);
+  rc = tp_configure(P, elem_bytes, 0, &warps, &smem, &fn);  // host-only: does the shape fit at all?
   if (rc != QKNORM_OK) return rc;
   const int tile = 32 >> P.log_g;
 
   const DeviceInfo* dev = nullptr;
   rc = current_device(&dev);
+  if (rc != QKNORM_OK) return rc;
+  rc = tp_configure(P, elem_bytes, dev->sm_count, &warps, &smem, &fn);
   if (rc != QKNORM_OK) return rc;
   if (smem > dev->smem_per_block) return QKNORM_ERR_SHAPE;
   rc = allow_dynamic_smem((const void*)fn, smem);
@@ -252,7 +261,7 @@ int launch_tile(const Params& P, const DeviceInfo& dev, cudaStream_t stream, boo
   r.inbox = reinterpret_cast<unsigned long long*>(dev.ring_error);  // only its status words are used
   int warps = 0, smem = 0;
   TpKernel fn = nullptr;
-  int rc = tp_configure(T, P.elem_bytes, &warps, &smem, &fn);
+  int rc = tp_configure(T, P.elem_bytes, dev.sm_count, &warps, &smem, &fn);
   if (rc != QKNORM_OK) return QKNORM_OK;  // does not fit: another variant takes the call
   if (smem > dev.smem_per_block) return QKNORM_OK;
   rc = allow_dynamic_smem((const void*)fn, smem);

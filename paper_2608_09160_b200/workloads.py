@@ -171,7 +171,7 @@ def small_parity_shapes() -> List[Workload]:
         ("s_24", 5, 24, 8, (1,)),
         ("s_unaligned", 7, 1001, 77, (1, 7)),
         ("s_149", 149, 5120, 1024, (1, 8)),
-        ("s_1025", 1025, 640, 128, (1, 4)),
+        ("s_2305", 2305, 640, 128, (1, 4)),
         ("s_8200", 33, 8200, 8200, (1, 5)),
         ("s_wide", 9, 16384, 2048, (1, 16)),
         ("s_max", 2, 65536, 8, (1,)),
@@ -179,17 +179,19 @@ def small_parity_shapes() -> List[Workload]:
         ("s_mha4", 257, 5120, 5120, (4,)),
         ("s_konly", 17, 0, 1024, (1, 4)),
         ("s_qonly", 17, 2048, 0, (1, 4)),
-        ("s_prefill_gqa", 1500, 5120, 1024, (8, 1)),     # warp-per-token kernel, several rows per warp
-        ("s_prefill_odd", 777, 1000, 136, (1,)),         # warp-per-token kernel, lanes with ragged chunk counts
-        ("s_prefill_s3", 650, 1536, 768, (3,)),          # shard count that leaves lanes idle
-        ("s_prefill_konly", 700, 0, 1024, (2,)),
-        ("s_prefill_s16", 640, 4096, 1024, (16,)),       # two lanes per shard, every lane issues a bulk copy
-        ("s_prefill_s5", 610, 2240, 560, (5, 7)),        # shard counts that are not powers of two
-        ("s_prefill_wide", 600, 16384, 4096, (1, 4)),    # rows too wide for one warp: the CTA-per-token TMA ring
+        ("s_prefill_gqa", 2500, 5120, 1024, (8, 1)),     # warp-per-token kernel, several rows per warp
+        ("s_prefill_odd", 2177, 1000, 136, (1,)),         # warp-per-token kernel, lanes with ragged chunk counts
+        ("s_prefill_s3", 2150, 1536, 768, (3,)),          # shard count that leaves lanes idle
+        ("s_prefill_konly", 2200, 0, 1024, (2,)),
+        ("s_prefill_s16", 2140, 4096, 1024, (16,)),       # two lanes per shard, every lane issues a bulk copy
+        ("s_prefill_s5", 2110, 2240, 560, (5, 7)),        # shard counts that are not powers of two
+        ("s_prefill_wide", 2100, 16384, 4096, (1, 4)),    # rows too wide for one warp: the CTA-per-token TMA ring
         ("s_tile_gqa", 3001, 1024, 128, (1,)),           # short unsharded rows: several tokens per warp, ragged last tile
-        ("s_tile_tiny", 1000, 64, 8, (1,)),              # 128-byte and 16-byte rows
-        ("s_tile_konly", 777, 0, 256, (1,)),
-        ("s_tile_qonly", 601, 1280, 0, (1,)),
+        ("s_tile_tiny", 2600, 64, 8, (1,)),              # 128-byte and 16-byte rows
+        ("s_tile_konly", 2277, 0, 256, (1,)),
+        ("s_tile_qonly", 2101, 1280, 0, (1,)),
+        ("s_mid_gqa", 1500, 5120, 1024, (1, 8)),         # a thousand-odd tokens: still the register-resident rows kernel
+        ("s_mid_mha", 1900, 2048, 2048, (2,)),
     ]
     out = []
     for i, (name, t, dq, dk, sh) in enumerate(shapes):

@@ -47,7 +47,7 @@ static int check(const uint16_t* y, size_t n, float want, const char* what) {
 }
 
 int main(void) {
-  const int64_t T = 700;
+  const int64_t T = 2100;
   const int32_t dq = 2048, dk = 512, S = 4;
   const float eps = 1e-6f, cq = 3.0f, ck = -0.5f, gq = 1.25f, gk = 2.0f;
   const size_t nq = (size_t)T * dq, nk = (size_t)T * dk;

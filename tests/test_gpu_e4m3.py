@@ -19,12 +19,12 @@ NTHREADS = max(1, min(32, os.cpu_count() or 1))
 SHAPES = [
     # name, T, dq, dk, shard counts, expected variant per shard count
     ("e_decode", 8, 4096, 4096, (1, 4), ("rows", "rows")),
-    ("e_gqa", 900, 5120, 1024, (8, 1), ("warp", "warp")),
-    ("e_mha", 700, 5120, 5120, (4,), ("warp",)),
+    ("e_gqa", 2300, 5120, 1024, (8, 1), ("warp", "warp")),
+    ("e_mha", 2100, 5120, 5120, (4,), ("warp",)),
     ("e_odd_width", 650, 1000, 136, (1,), ("general",)),          # not a multiple of 16 elements
-    ("e_ragged", 777, 1008, 144, (1, 3), ("tile", "warp")),       # multiples of 16, ragged over the lanes
+    ("e_ragged", 2177, 1008, 144, (1, 3), ("tile", "warp")),       # multiples of 16, ragged over the lanes
     ("e_tiny", 3, 16, 16, (1,), ("rows",)),
-    ("e_konly", 600, 0, 2048, (2,), ("warp",)),
+    ("e_konly", 2100, 0, 2048, (2,), ("warp",)),
 ]
 
 
@@ -132,7 +132,7 @@ def test_full_size_e4m3(libqknorm, name):
 def test_e4m3_gamma_outside_fp16_takes_the_bf16_gamma_path(libqknorm, dq, dk, variant):
     """The prefill kernels keep an fp16 copy of gamma when every value fits fp16; one value that
     does not (2^-20, 1e5) must switch the whole call to the bf16-gamma arithmetic with the same result."""
-    w = W.Workload("e_wide_gamma", tokens=700, dq=dq, dk=dk, shards=(1,), seed=31, sigma=1.5)
+    w = W.Workload("e_wide_gamma", tokens=2200, dq=dq, dk=dk, shards=(1,), seed=31, sigma=1.5)
     inp = W.make_inputs_e4m3(w)
     gq = inp["gamma_q"].clone()
     gq[5] = 2.0 ** -20

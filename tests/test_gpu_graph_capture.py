@@ -12,7 +12,7 @@ from tests import gpu_harness as H
 pytestmark = pytest.mark.gpu
 
 CASES = [("decode", 8, 4096, 4096, 1, "rows"), ("decode-sharded", 64, 4096, 4096, 4, "rows"),
-         ("prefill-sharded", 700, 5120, 1024, 8, "warp")]
+         ("prefill-sharded", 2100, 5120, 1024, 8, "warp")]
 
 
 @pytest.mark.parametrize("name,T,dq,dk,S,variant", CASES, ids=[c[0] for c in CASES])

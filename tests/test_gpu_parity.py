@@ -120,11 +120,11 @@ def test_unaligned_buffers_take_the_general_kernel(libqknorm, skew):
 
 
 @pytest.mark.parametrize("name,S,variant", [
-    ("s_t1", 1, "rows"), ("s_149", 8, "rows"), ("s_gqa8", 8, "rows"),          # few tokens: register-resident rows
+    ("s_t1", 1, "rows"), ("s_149", 8, "rows"), ("s_gqa8", 8, "rows"), ("s_mid_gqa", 1, "rows"), ("s_mid_mha", 2, "rows"),          # few tokens: register-resident rows
     ("s_prefill_gqa", 8, "warp"), ("s_prefill_gqa", 1, "warp"), ("s_prefill_odd", 1, "tile"),
-    ("s_1025", 1, "tile"), ("s_tile_gqa", 1, "tile"), ("s_tile_tiny", 1, "tile"), ("s_tile_konly", 1, "tile"),
+    ("s_2305", 1, "tile"), ("s_tile_gqa", 1, "tile"), ("s_tile_tiny", 1, "tile"), ("s_tile_konly", 1, "tile"),
     ("s_tile_qonly", 1, "tile"),                                               # short unsharded rows: several tokens per warp
-    ("s_prefill_s3", 3, "warp"), ("s_prefill_konly", 2, "warp"), ("s_1025", 4, "warp"),
+    ("s_prefill_s3", 3, "warp"), ("s_prefill_konly", 2, "warp"), ("s_2305", 4, "warp"),
     ("s_prefill_s16", 16, "warp"), ("s_prefill_s5", 5, "warp"),
     ("s_prefill_wide", 1, "ring"), ("s_prefill_wide", 4, "ring"),
     ("s_unaligned", 7, "general"), ("s_max", 1, "general"),

@@ -194,3 +194,34 @@ def test_argument_errors_launch_nothing(libqknorm):
         tp.qknorm_fwd_tp(bufs, N, T, w.eps, 1)
     assert ei.value.status == binding.QKNORM_ERR_ALIAS
     assert binding.launch_count() == n0
+
+
+def _random_tp_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    for i in range(n):
+        N = int(rng.choice([1, 2, 3, 4, 5, 8, 12, 16]))
+        wq = int(rng.integers(1, 160)) * 8 if rng.integers(0, 6) else 0
+        wk = int(rng.integers(1, 96)) * 8 if (wq == 0 or rng.integers(0, 5)) else 0
+        while (wq + wk) * N > 20000 or wq * N > 65536:      # keep the oracle quick
+            wq, wk = wq // 2 // 8 * 8, max(8, wk // 2 // 8 * 8)
+        T = int(rng.integers(1, 3000))
+        cases.append((i, N, T, wq, wk))
+    return cases
+
+
+RANDOM_TP = _random_tp_cases(16, seed=31)
+
+
+@pytest.mark.parametrize("i,N,T,wq,wk", RANDOM_TP, ids=[f"tp{c[0]}-N{c[1]}-T{c[2]}-{c[3]}+{c[4]}" for c in RANDOM_TP])
+def test_random_tensor_parallel_shapes(libqknorm, i, N, T, wq, wk):
+    w = W.Workload(f"tp_rand{i}", tokens=T, dq=wq * N, dk=wk * N, shards=(N,), seed=7000 + i, sigma=(0.5, 2.0)[i % 2])
+    inp = W.make_inputs(w)
+    dev = device_slices(inp, N)
+    grp = tp.EmulatedGroup(N, token_capacity=T + i)
+    for _ in range(2):                     # two calls in a row on the same inboxes
+        bufs = grp.buffers(dev["q"], dev["k"], dev["gamma_q"], dev["gamma_k"], stats=True)
+        grp.forward(bufs, w.eps)
+        torch.cuda.synchronize()
+        check_group(bufs, oracle_sharded(inp, N, w.eps), f"random tp {i}")
+    assert all(tp.status(b)["status"] == tp.STATUS_OK for b in grp.inboxes)

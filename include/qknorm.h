@@ -129,6 +129,13 @@ int qknorm_fwd_strided(const void* q, const void* k, const void* gamma_q, const 
                        int64_t tokens, int32_t dq, int32_t dk, int64_t ld_q, int64_t ld_k, float eps,
                        void* out_q, void* out_k, int64_t ld_out_q, int64_t ld_out_k, void* stream);
 
+/* qknorm_fwd_strided with FP8-E4M3 activations (one byte per element, gamma bf16; see
+ * qknorm_fwd_e4m3).  Strides are in elements; the vectorised kernels need every ld to be a
+ * multiple of 16 elements. */
+int qknorm_fwd_strided_e4m3(const void* q, const void* k, const void* gamma_q, const void* gamma_k,
+                            int64_t tokens, int32_t dq, int32_t dk, int64_t ld_q, int64_t ld_k, float eps,
+                            void* out_q, void* out_k, int64_t ld_out_q, int64_t ld_out_k, void* stream);
+
 /*
  * qknorm_fwd_headwise -- the other granularity Section II-A names: "headwise QK-Norm
  * computes an independent factor for each attention head".  Row t of q is cut into

@@ -24,6 +24,7 @@ EXPORTS = (
     "qknorm_fwd_sharded_ex",
     "qknorm_fwd_e4m3",
     "qknorm_fwd_strided",
+    "qknorm_fwd_strided_e4m3",
     "qknorm_fwd_headwise",
     "qknorm_baseline_gather_then_norm",
     "qknorm_baseline_two_pass",
@@ -87,6 +88,8 @@ def load() -> ctypes.CDLL:
     lib.qknorm_fwd_sharded_e4m3.restype = ctypes.c_int
     lib.qknorm_fwd_strided.argtypes = [_vp, _vp, _vp, _vp, i64, i32, i32, i64, i64, f32, _vp, _vp, i64, i64, _vp]
     lib.qknorm_fwd_strided.restype = ctypes.c_int
+    lib.qknorm_fwd_strided_e4m3.argtypes = lib.qknorm_fwd_strided.argtypes
+    lib.qknorm_fwd_strided_e4m3.restype = ctypes.c_int
     lib.qknorm_fwd_headwise.argtypes = [_vp, _vp, _vp, _vp, i64, i32, i32, i32, i64, i64, f32, _vp, _vp, i64, i64,
                                         _vp, _vp, _vp]
     lib.qknorm_fwd_headwise.restype = ctypes.c_int
@@ -309,28 +312,31 @@ def qknorm_fwd_sharded(q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps: 
     return out_q_shards, out_k_shards
 
 
-def _expect_rows(t: Optional[torch.Tensor], T: int, d: int, what: str) -> int:
-    """A [T, d] bf16 CUDA view whose rows are contiguous; returns its row stride in elements."""
+def _expect_rows(t: Optional[torch.Tensor], T: int, d: int, what: str, dtype=torch.bfloat16) -> int:
+    """A [T, d] CUDA view of `dtype` whose rows are contiguous; returns its row stride in elements."""
     if t is None:
         raise QKNormError(QKNORM_ERR_NULL, f"{what} is None")
-    if (not t.is_cuda or t.dtype != torch.bfloat16 or tuple(t.shape) != (T, d)
+    if (not t.is_cuda or t.dtype != dtype or tuple(t.shape) != (T, d)
             or (d > 1 and t.stride(1) != 1)):
-        raise QKNormError(QKNORM_ERR_SHAPE, f"{what}: expected a bf16 CUDA [{T}, {d}] view with unit column stride")
+        raise QKNormError(QKNORM_ERR_SHAPE, f"{what}: expected a {dtype} CUDA [{T}, {d}] view with unit column stride")
     return int(t.stride(0)) if T > 1 else d
 
 
 def qknorm_fwd_strided(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=None, *, stream=None):
     """qknorm_fwd_strided: q [T,dq] and k [T,dk] may be column blocks of a wider buffer
-    (row stride taken from the tensors); out_* default to the inputs (in place)."""
+    (row stride taken from the tensors); out_* default to the inputs (in place).  bf16, or
+    float8_e4m3fn activations (qknorm_fwd_strided_e4m3)."""
     lib = load()
     T, dq, dk = q.shape[0], q.shape[1], k.shape[1]
+    cfunc = lib.qknorm_fwd_strided_e4m3 if q.dtype is torch.float8_e4m3fn else lib.qknorm_fwd_strided
     out_q = q if out_q is None else out_q
     out_k = k if out_k is None else out_k
-    ld = [_expect_rows(q, T, dq, "q"), _expect_rows(k, T, dk, "k"),
-          _expect_rows(out_q, T, dq, "out_q"), _expect_rows(out_k, T, dk, "out_k")]
+    act = q.dtype if q.dtype is torch.float8_e4m3fn else torch.bfloat16
+    ld = [_expect_rows(q, T, dq, "q", act), _expect_rows(k, T, dk, "k", act),
+          _expect_rows(out_q, T, dq, "out_q", act), _expect_rows(out_k, T, dk, "out_k", act)]
     _expect(gamma_q, (dq,), torch.bfloat16, "gamma_q")
     _expect(gamma_k, (dk,), torch.bfloat16, "gamma_k")
-    _invoke(lib.qknorm_fwd_strided, [_ptr(q), _ptr(k), _ptr(gamma_q), _ptr(gamma_k), T, dq, dk, ld[0], ld[1],
+    _invoke(cfunc, [_ptr(q), _ptr(k), _ptr(gamma_q), _ptr(gamma_k), T, dq, dk, ld[0], ld[1],
                                      float(eps), _ptr(out_q), _ptr(out_k), ld[2], ld[3]], stream,
             (q, k, gamma_q, gamma_k, out_q, out_k))
     return out_q, out_k

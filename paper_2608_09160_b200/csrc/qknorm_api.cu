@@ -892,6 +892,15 @@ int qknorm_fwd_strided(const void* q, const void* k, const void* gamma_q, const 
                      nullptr, nullptr, stream, ld);
 }
 
+int qknorm_fwd_strided_e4m3(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
+                            int32_t dq, int32_t dk, int64_t ld_q, int64_t ld_k, float eps, void* out_q, void* out_k,
+                            int64_t ld_out_q, int64_t ld_out_k, void* stream) {
+  if (ld_q < 0 || ld_k < 0 || ld_out_q < 0 || ld_out_k < 0) return QKNORM_ERR_SHAPE;
+  const int64_t ld[4] = {ld_q, ld_k, ld_out_q, ld_out_k};
+  return qknorm::run(1, &q, &k, &gamma_q, &gamma_k, 1, tokens, dq, dk, eps, &out_q, &out_k, nullptr, nullptr,
+                     nullptr, nullptr, stream, ld);
+}
+
 int qknorm_fwd_headwise(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
                         int32_t dq, int32_t dk, int32_t head_dim, int64_t ld_q, int64_t ld_k, float eps,
                         void* out_q, void* out_k, int64_t ld_out_q, int64_t ld_out_k, float* rstd_q,

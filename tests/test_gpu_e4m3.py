@@ -146,3 +146,25 @@ def test_e4m3_gamma_outside_fp16_takes_the_bf16_gamma_path(libqknorm, dq, dk, va
     compare_e4m3(W.e4m3_bits(oq.cpu()), ref_q, "wide gamma q")
     compare_e4m3(W.e4m3_bits(ok.cpu()), ref_k, "wide gamma k")
     assert (W.e4m3_bits(oq.cpu())[:, 77] & 0x7F == 0x7E).mean() > 0.5     # 1e5 * x saturates
+
+
+@pytest.mark.parametrize("T,dq,dk,pad,variant", [(2200, 4096, 1024, 0, "warp"), (2300, 1024, 256, 16, "tile"),
+                                                  (40, 2048, 512, 32, "rows")])
+def test_e4m3_rows_strided_inside_a_fused_qkv_buffer(libqknorm, T, dq, dk, pad, variant):
+    """FP8 rows that are column blocks of one fused [T, dq + 2*dk (+ pad)] buffer, normalised in place;
+    the V block and the padding keep their bytes."""
+    w = W.Workload("e_qkv", tokens=T, dq=dq, dk=dk, shards=(1,), seed=600 + T, sigma=1.5)
+    inp = W.make_inputs_e4m3(w)
+    ld = dq + 2 * dk + pad
+    buf = torch.full((T, ld), 0x55, dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn)
+    buf[:, :dq] = inp["q"].cuda()
+    buf[:, dq:dq + dk] = inp["k"].cuda()
+    q, k = buf[:, :dq], buf[:, dq:dq + dk]
+    binding.qknorm_fwd_strided(q, k, inp["gamma_q"].cuda(), inp["gamma_k"].cuda(), w.eps)
+    torch.cuda.synchronize()
+    assert binding.last_variant() == variant
+    host = buf.cpu()
+    for nm, sl in (("q", slice(0, dq)), ("k", slice(dq, dq + dk))):
+        ref = oracle.rmsnorm_e4m3([W.e4m3_bits(inp[nm])], [W.bf16_bits(inp["gamma_" + nm])], w.eps)
+        compare_e4m3(W.e4m3_bits(host[:, sl].contiguous()), ref["y"][0], f"strided e4m3 {nm}")
+    assert bool((host[:, dq + dk:].contiguous().view(torch.uint8) == 0x55).all())

@@ -26,6 +26,10 @@
  *  - Asynchrony: work is enqueued on `stream` (a cudaStream_t passed as void*;
  *    NULL = the legacy default stream) and the call returns without
  *    synchronising.  No cudaMalloc, no cudaMemcpy, no host synchronisation.
+ *    Calls of up to about two thousand tokens are launched with programmatic stream
+ *    serialisation: the launch may begin while the previous kernel of the stream is still
+ *    running, and the kernel waits for that kernel to complete (and its writes to be
+ *    visible) before its first memory access, so stream order is kept as usual.
  *  - Errors: the return value is a qknorm_status.  On any error nothing has
  *    been launched.  tokens == 0 returns QKNORM_OK without a launch.
  *  - A tensor can be skipped: dq == 0 (with its pointers ignored) means "K

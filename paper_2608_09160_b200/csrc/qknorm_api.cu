@@ -519,7 +519,24 @@ int launch(Params& P, cudaStream_t stream) {
       long long grid = (long long)bres * sms;  // bounded grid of co-resident CTAs
       if (grid > P.T) grid = P.T;
       apply_plan(P, plan);
-      fn<<<(unsigned)grid, plan.threads, 0, stream>>>(P);
+      if (env_int("QKNORM_PDL", 1)) {
+        // allow this launch to begin while the previous kernel of the stream is still running; the
+        // kernel itself waits for that kernel's completion before its first memory access
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(plan.threads);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, fn, P);
+        if (e != cudaSuccess) return set_cuda_error(e);
+      } else {
+        fn<<<(unsigned)grid, plan.threads, 0, stream>>>(P);
+      }
       return finish_launch("rows");
     }
   }

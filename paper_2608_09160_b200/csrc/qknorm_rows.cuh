@@ -18,7 +18,13 @@ namespace qknorm {
 template <int N, class IO>
 __global__ void __launch_bounds__(max_threads_for(N), min_blocks_for(N)) rows_kernel(const __grid_constant__ Params P) {
   __shared__ __align__(16) float slots[2][kMaxSlots];
+  // Programmatic dependent launch (both instructions are no-ops without the launch attribute): let
+  // the next kernel of the stream begin its own launch now, work out this thread's place in the row,
+  // and only then wait: no memory is touched before everything earlier in the stream has completed
+  // and is visible.  Back-to-back decode calls overlap their launch latencies this way.
+  asm volatile("griddepcontrol.launch_dependents;");
   const LaneMap m = make_lane<IO>(P, threadIdx.x, N);
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   uint4 gm[N * IO::kGammaVecs];
   load_gamma<IO, N>(m, gm);
 

@@ -48,3 +48,33 @@ def test_capture_and_replay_with_new_inputs(libqknorm, name, T, dq, dk, S, varia
         H.compare_output(H.bits(W.unshard_columns([t.cpu() for t in oq])), ref["q"]["y"], f"{name} replay q")
         H.compare_output(H.bits(W.unshard_columns([t.cpu() for t in ok])), ref["k"]["y"], f"{name} replay k")
     assert binding.device_error_word() == 0
+
+
+def test_stream_order_is_kept_when_launches_overlap(libqknorm):
+    """Decode-size calls may begin their launch while the previous kernel of the stream still runs.
+    A chain of dependent work without any synchronisation in between -- another kernel rewrites the
+    input, the call normalises it in place, the next call normalises that result again -- must still
+    see every predecessor's writes."""
+    w = W.Workload("chain", tokens=48, dq=4096, dk=1024, shards=(1,), seed=55, sigma=3.0)
+    inp = W.make_inputs(w)
+    q, k = inp["q"].cuda(), inp["k"].cuda()
+    gq, gk = inp["gamma_q"].cuda(), inp["gamma_k"].cuda()
+    src_q, src_k = q.clone(), k.clone()
+    call = binding.prepared(binding.qknorm_fwd, q, k, gq, gk, w.eps, q, k)
+    call()                             # one pass on its own, synchronised: what the second pass starts from
+    torch.cuda.synchronize()
+    once = {"q": q.cpu(), "k": k.cpu(), "gamma_q": inp["gamma_q"], "gamma_k": inp["gamma_k"]}
+    H.compare_output(H.bits(q), H.oracle_unsharded(inp, w.eps)["q"]["y"], "first pass q")
+    for i in range(40):
+        q.copy_(src_q)                 # a foreign kernel writes the input ...
+        k.copy_(src_k)
+        if i % 2:
+            q.neg_()                   # ... a second one changes it again ...
+        call()                         # ... and two library calls in a row consume it, the second the first's output
+        call()
+    torch.cuda.synchronize()
+    assert binding.last_variant() == "rows"
+    ref2 = H.oracle_unsharded(once, w.eps)
+    want_q = ref2["q"]["y"] ^ np.uint16(0x8000)          # the last round (i = 39) negated q first
+    H.compare_output(H.bits(q), want_q, "chained q")
+    H.compare_output(H.bits(k), ref2["k"]["y"], "chained k")

@@ -129,6 +129,18 @@ int qknorm_tp_status(const void* inbox, int32_t* out);
 int qknorm_tp_clear_status(void* inbox, void* stream);
 
 /*
+ * qknorm_tp_slot_index -- position (in 64-bit words from the start of an inbox) of the slot that
+ * holds source rank `src_rank`'s scalar of token 0 for a call with this epoch; token t is t words
+ * further.  tensor: 0 = Q, 1 = K.  Returns -1 for arguments out of range.
+ * qknorm_tp_inbox_peek / _poke -- synchronous copies of n_words 64-bit words between an inbox (from
+ * word first_word) and HOST memory: for tests, inspection and recovery tools (a slot is
+ * (uint64_t)epoch << 32 | fp32 bits).  Not for use while a call on the inbox is in flight.
+ */
+int64_t qknorm_tp_slot_index(int32_t num_ranks, int64_t token_capacity, uint32_t epoch, int32_t tensor, int32_t src_rank);
+int qknorm_tp_inbox_peek(const void* inbox, int64_t first_word, int64_t n_words, uint64_t* out);
+int qknorm_tp_inbox_poke(void* inbox, int64_t first_word, int64_t n_words, const uint64_t* in);
+
+/*
  * Inbox management for one process per GPU.  These are the only routines of the
  * library that allocate or map device memory, and none of them is called by the
  * forward entry points.

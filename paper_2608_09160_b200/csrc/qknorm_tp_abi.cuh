@@ -31,6 +31,28 @@ int qknorm_tp_status(const void* inbox, int32_t* out) {
   return QKNORM_OK;
 }
 
+int64_t qknorm_tp_slot_index(int32_t num_ranks, int64_t token_capacity, uint32_t epoch, int32_t tensor, int32_t src_rank) {
+  if (num_ranks < 1 || num_ranks > qknorm::kMaxShards || token_capacity < 1 || epoch == 0u) return -1;
+  if (tensor < 0 || tensor > 1 || src_rank < 0 || src_rank >= num_ranks) return -1;
+  return (int64_t)qknorm::tp_slot_index((int)(epoch & 1u), tensor, src_rank, num_ranks, token_capacity);
+}
+
+int qknorm_tp_inbox_peek(const void* inbox, int64_t first_word, int64_t n_words, uint64_t* out) {
+  if (!inbox || !out) return QKNORM_ERR_NULL;
+  if (first_word < 0 || n_words < 0) return QKNORM_ERR_SHAPE;
+  cudaError_t e = cudaMemcpy(out, (const unsigned long long*)inbox + first_word, (size_t)n_words * 8, cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  return QKNORM_OK;
+}
+
+int qknorm_tp_inbox_poke(void* inbox, int64_t first_word, int64_t n_words, const uint64_t* in) {
+  if (!inbox || !in) return QKNORM_ERR_NULL;
+  if (first_word < 0 || n_words < 0) return QKNORM_ERR_SHAPE;
+  cudaError_t e = cudaMemcpy((unsigned long long*)inbox + first_word, in, (size_t)n_words * 8, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return qknorm::set_cuda_error(e);
+  return QKNORM_OK;
+}
+
 int qknorm_tp_clear_status(void* inbox, void* stream) {
   if (!inbox) return QKNORM_ERR_NULL;
   cudaError_t e = cudaMemsetAsync(inbox, 0, 8 * qknorm::kTpHeaderWords, (cudaStream_t)stream);

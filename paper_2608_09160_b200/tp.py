@@ -30,6 +30,9 @@ EXPORTS = (
     "qknorm_fwd_tp_e4m3",
     "qknorm_tp_status",
     "qknorm_tp_clear_status",
+    "qknorm_tp_slot_index",
+    "qknorm_tp_inbox_peek",
+    "qknorm_tp_inbox_poke",
     "qknorm_tp_inbox_create",
     "qknorm_tp_inbox_zero",
     "qknorm_tp_inbox_destroy",
@@ -70,6 +73,9 @@ def lib() -> ctypes.CDLL:
         fn.argtypes = [ctypes.POINTER(CTpRank), i32, i32, i64, i64, i32, i32, ctypes.POINTER(i64), f32, u32, u32, _vp]
     L.qknorm_tp_status.argtypes = [_vp, ctypes.POINTER(i32)]
     L.qknorm_tp_clear_status.argtypes = [_vp, _vp]
+    L.qknorm_tp_slot_index.argtypes = [i32, i64, u32, i32, i32]
+    L.qknorm_tp_inbox_peek.argtypes = [_vp, i64, i64, ctypes.POINTER(ctypes.c_uint64)]
+    L.qknorm_tp_inbox_poke.argtypes = [_vp, i64, i64, ctypes.POINTER(ctypes.c_uint64)]
     L.qknorm_tp_inbox_create.argtypes = [i32, i64, ctypes.POINTER(_vp)]
     L.qknorm_tp_inbox_zero.argtypes = [_vp, i32, i64, _vp]
     L.qknorm_tp_inbox_destroy.argtypes = [_vp]
@@ -78,6 +84,7 @@ def lib() -> ctypes.CDLL:
     L.qknorm_tp_ipc_close.argtypes = [_vp]
     for name in EXPORTS:
         getattr(L, name).restype = ctypes.c_int
+    L.qknorm_tp_slot_index.restype = ctypes.c_int64
     _ready = True
     return L
 
@@ -196,6 +203,29 @@ def status(inbox) -> dict:
     out = (ctypes.c_int32 * 4)()
     _check(lib().qknorm_tp_status(_addr(inbox), out))
     return {"status": out[0], "token": out[1], "missing_rank": out[2]}
+
+
+def slot_index(num_ranks: int, token_capacity: int, epoch: int, tensor: int, src_rank: int) -> int:
+    """Word offset of source rank `src_rank`'s slot for token 0 (tensor 0 = Q, 1 = K) in an inbox."""
+    i = lib().qknorm_tp_slot_index(num_ranks, token_capacity, epoch, tensor, src_rank)
+    if i < 0:
+        raise QKNormError(binding.QKNORM_ERR_SHAPE, "slot index arguments out of range")
+    return i
+
+
+def peek(inbox, first_word: int, n_words: int):
+    """n_words 64-bit words of an inbox as a numpy uint64 array (synchronous)."""
+    import numpy as np
+    out = np.empty(n_words, dtype=np.uint64)
+    _check(lib().qknorm_tp_inbox_peek(_addr(inbox), first_word, n_words, out.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64))))
+    return out
+
+
+def poke(inbox, first_word: int, words) -> None:
+    """Writes a numpy uint64 array into an inbox from word first_word on (synchronous)."""
+    import numpy as np
+    w = np.ascontiguousarray(words, dtype=np.uint64)
+    _check(lib().qknorm_tp_inbox_poke(_addr(inbox), first_word, w.size, w.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64))))
 
 
 def clear_status(inbox, stream=None) -> None:

@@ -213,6 +213,11 @@ tp_kernel(const __grid_constant__ TpParams P) {
   }
   const uint32_t row_bytes = ((uint32_t)P.wq + (uint32_t)P.wk) * IO::kBytes;
   const uint64_t policy = ptx::policy_evict_first();
+  // Short rows (up to 1 KB) that follow one another without a gap both in memory and in the stage:
+  // the whole tile of that tensor is ONE bulk copy (issued by the lane of its first row) instead of
+  // one per row.  Measured: 320-byte FP8 rows 3.9 -> 4.8 TB/s; rows of 2 KB are faster copied singly.
+  const bool whole_tile = my_bytes != 0 && my_bytes <= 1024u && my_pitch == my_bytes &&
+                          (issue_q ? (uint32_t)P.q_row_stride : (uint32_t)P.k_row_stride) == my_bytes;
 
   const int cta_warps = blockDim.x >> 5;
   const long long first = (cta * cta_warps + warp) * tile;
@@ -224,9 +229,14 @@ tp_kernel(const __grid_constant__ TpParams P) {
     const uint32_t bar = bar0 + 8u * (uint32_t)st;
     if (lane == 0) ptx::mbar_arrive_expect_tx(bar, (uint32_t)n * row_bytes);
     __syncwarp();
-    if (my_bytes && is < n)
+    if (whole_tile) {
+      if (is == 0)
+        ptx::bulk_load(stages0 + (uint32_t)st * (uint32_t)P.stage_bytes + my_dst,
+                       my_src + (unsigned long long)t0 * my_pitch, (uint32_t)n * my_bytes, bar, policy);
+    } else if (my_bytes && is < n) {
       ptx::bulk_load(stages0 + (uint32_t)st * (uint32_t)P.stage_bytes + my_dst,
                      my_src + (unsigned long long)(t0 + is) * my_pitch, my_bytes, bar, policy);
+    }
   };
   __syncwarp();
   if (n_tiles > 0) arm(first, 0);

@@ -42,7 +42,8 @@ int tp_configure(TpParams& P, int elem_bytes, int sm_count, int* warps_out, int*
     P.log_g = log_g;
     // rows of a tile side by side in the stage; the skew keeps lane groups that read in the same
     // quarter-warp on different banks
-    const int skew = (tile > 1 && g < 8) ? g * 16 : 0;
+    const bool contiguous = P.ldxq == wq && P.ldxk == wk && env_int("QKNORM_TP_BULK", 1) != 0;
+    const int skew = (tile > 1 && g < 8 && !contiguous) ? g * 16 : 0;  // contiguous rows: one copy per tile instead
     P.q_row_stride = cq ? wq * elem_bytes + skew : 0;
     P.k_row_stride = ck ? wk * elem_bytes + skew : 0;
     P.k_base = tile * P.q_row_stride;

@@ -209,8 +209,21 @@ bool vector_path_ok(const Params& P) {
   return true;
 }
 
+// The experiment knobs (QKNORM_FORCE_VARIANT, QKNORM_WARPS, ...) are looked at only in a process that
+// was started with QKNORM_DEBUG_ENV set: a production process makes no getenv call per launch and
+// cannot be steered by a stray variable.
+bool debug_env_enabled() {
+  static const bool on = [] {
+    const char* v = getenv("QKNORM_DEBUG_ENV");
+    return v != nullptr && *v != '\0' && *v != '0';
+  }();
+  return on;
+}
+
+const char* env_str(const char* name) { return debug_env_enabled() ? getenv(name) : nullptr; }
+
 int env_int(const char* name, int fallback) {
-  const char* v = getenv(name);
+  const char* v = env_str(name);
   if (!v || !*v) return fallback;
   return atoi(v);
 }
@@ -472,7 +485,7 @@ int launch(Params& P, cudaStream_t stream) {
   int rc = current_device(&dev);
   if (rc != QKNORM_OK) return rc;
   const int sms = dev->sm_count;
-  const char* force = getenv("QKNORM_FORCE_VARIANT");
+  const char* force = env_str("QKNORM_FORCE_VARIANT");
   const bool force_general = force && strcmp(force, "general") == 0;
   const bool force_rows = force && strcmp(force, "rows") == 0;
   const bool force_ring = force && strcmp(force, "ring") == 0;
@@ -765,7 +778,7 @@ int run_headwise(const void* q, const void* k, const void* gq, const void* gk, i
     hs[i]->ldy = ts[i]->ldy * 2;
     hs[i]->nh = ts[i]->d / head_dim;
   }
-  const char* force = getenv("QKNORM_FORCE_VARIANT");
+  const char* force = env_str("QKNORM_FORCE_VARIANT");
   const bool vec = !(force && strcmp(force, "general") == 0) && head_dim % 8 == 0 && head_dim <= 256 && vector_path_ok(P);
   if (vec) {
     H.hc = head_dim / 8;

@@ -1,6 +1,10 @@
 import os
 import sys
 
+# the tests steer kernel variants through the library's experiment knobs, which it only reads
+# in a process started with this variable set
+os.environ.setdefault("QKNORM_DEBUG_ENV", "1")
+
 import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))

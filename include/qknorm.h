@@ -43,7 +43,9 @@
  *    reproducible run to run (no atomics).
  *  - Fast path: when every base pointer is 16-byte aligned and every (shard)
  *    width is a multiple of 8 elements, vectorised kernels run; any other
- *    width or alignment is served by a slower general kernel, not an error.
+ *    width or alignment is served by a slower general kernel, not an error.  A call is
+ *    one kernel launch, except when Q and K together are wider than 32768 elements and
+ *    each fits alone: then Q and K (whose statistics are independent) get a launch each.
  */
 #ifndef QKNORM_H_
 #define QKNORM_H_

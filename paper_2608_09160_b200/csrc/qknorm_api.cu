@@ -552,6 +552,19 @@ int launch(Params& P, cudaStream_t stream) {
       }
       return finish_launch("rows");
     }
+    // Q and K together are too wide for one CTA's registers (more than 32768 elements): the two
+    // statistics are independent, so each tensor gets its own launch if it fits alone.
+    if (P.q.d != 0 && P.k.d != 0) {
+      Params Q = P, K = P;
+      memset(&Q.k, 0, sizeof(Q.k));
+      memset(&K.q, 0, sizeof(K.q));
+      RowsPlan pq, pk;
+      if (plan_rows(Q, false, &pq) && plan_rows(K, false, &pk)) {
+        rc = launch(Q, stream);
+        if (rc != QKNORM_OK) return rc;
+        return launch(K, stream);
+      }
+    }
   }
   void (*gen)(const Params) = P.elem_bytes == 1 ? general_kernel<IoE4m3> : general_kernel<IoBf16>;
   int bres = 1;

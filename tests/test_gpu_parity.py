@@ -268,3 +268,16 @@ def test_tiny_and_subnormal_inputs_are_not_flushed(libqknorm, T):
     got = H.bits(oq)
     H.compare_output(got, ref, f"tiny inputs T={T}")
     assert (got[0] & 0x7FFF).any(), "subnormal inputs were flushed to zero"
+
+
+@pytest.mark.parametrize("T,S,variant", [(40, 1, "rows"), (2100, 4, "warp")])   # variant of the second (K) launch
+def test_rows_too_wide_for_one_cta_take_one_launch_per_tensor(libqknorm, T, S, variant):
+    """Q and K together beyond 32768 elements do not fit one CTA's registers; each fits alone, and the
+    two statistics are independent, so the call is served by two launches of the vectorised kernels
+    instead of the slow general one."""
+    w = W.Workload("very_wide", tokens=T, dq=32768, dk=8192, shards=(S,), seed=321, sigma=0.5)
+    n0 = binding.launch_count()
+    res = run_case(w, S, in_place=True)
+    assert binding.launch_count() == n0 + 2
+    assert res["variant"] == variant
+    check_against_oracle(w, S, res)

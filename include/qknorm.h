@@ -44,8 +44,9 @@
  *  - Fast path: when every base pointer is 16-byte aligned and every (shard)
  *    width is a multiple of 8 elements, vectorised kernels run; any other
  *    width or alignment is served by a slower general kernel, not an error.  A call is
- *    one kernel launch, except when Q and K together are wider than 32768 elements and
- *    each fits alone: then Q and K (whose statistics are independent) get a launch each.
+ *    one kernel launch, except for some very wide rows (Q and K together beyond 32768
+ *    elements, or beyond 10240 elements in 8 or more slices with K much narrower than Q):
+ *    there Q and K, whose statistics are independent, get a launch each.
  */
 #ifndef QKNORM_H_
 #define QKNORM_H_

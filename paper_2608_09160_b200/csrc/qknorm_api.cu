@@ -407,6 +407,15 @@ int launch_ring(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   return rc;
 }
 
+// Chunk slots per lane the warp-per-token kernel would need for this call.
+int warp_slots_needed(const Params& P) {
+  int log_g = 5;
+  while ((P.S << log_g) > 32) --log_g;
+  const int g = 1 << log_g;
+  const int cq = P.q.d ? P.q.w * P.elem_bytes / 16 : 0, ck = P.k.d ? P.k.w * P.elem_bytes / 16 : 0;
+  return round_up((cq + g - 1) / g, 4) + (ck + g - 1) / g;
+}
+
 // The warp-per-token kernel (prefill sizes, gathered rows of up to 40 chunks per lane).
 int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* done) {
   *done = false;
@@ -515,6 +524,20 @@ int launch(Params& P, cudaStream_t stream) {
       bool done = false;
       rc = launch_warp(P, *dev, stream, &done);
       if (rc != QKNORM_OK || done) return rc;
+    }
+    // Rows too wide for the warp kernel, cut into 8 or more slices, K much narrower than Q (a large
+    // GQA layer under 8-way tensor parallelism): the CTA-per-token layout spends a lane group on every
+    // narrow K slice.  Q and K have independent statistics, so each gets its own launch -- Q on the
+    // ring kernel, K on the warp kernel.  Measured (16384 + 2048 wide, 8 slices, 8138 tokens): 154 us
+    // in one launch, 114 us in two.
+    if (!latency && !force && P.q.d != 0 && P.k.d != 0 && P.S >= 8 && P.k.d * 4 <= P.q.d &&
+        warp_round_up_l(warp_slots_needed(P)) < 0) {
+      Params Q = P, K = P;
+      memset(&Q.k, 0, sizeof(Q.k));
+      memset(&K.q, 0, sizeof(K.q));
+      rc = launch(Q, stream);
+      if (rc != QKNORM_OK) return rc;
+      return launch(K, stream);
     }
     if (!latency && !force_rows) {
       bool done = false;

@@ -281,3 +281,14 @@ def test_rows_too_wide_for_one_cta_take_one_launch_per_tensor(libqknorm, T, S, v
     assert binding.launch_count() == n0 + 2
     assert res["variant"] == variant
     check_against_oracle(w, S, res)
+
+
+def test_wide_gqa_rows_in_eight_slices_take_one_launch_per_tensor(libqknorm):
+    """Rows too wide for the warp kernel with K much narrower than Q and 8 slices: Q goes to the ring
+    kernel and K to the warp kernel, two launches, same results (statistics, partials included)."""
+    w = W.Workload("wide_gqa", tokens=2100, dq=16384, dk=2048, shards=(8,), seed=322)
+    n0 = binding.launch_count()
+    res = run_case(w, 8)
+    assert binding.launch_count() == n0 + 2
+    assert res["variant"] == "warp"          # of the second (K) launch
+    check_against_oracle(w, 8, res)

@@ -270,7 +270,7 @@ int qknorm_last_cuda_error(void);
 int qknorm_device_error_word(int* out);
 
 /* Name of the kernel variant the last successful call on this thread launched
- * ("warp", "tile", "ring", "rows", "general", "head", "head_general", "two_pass", "tp", "none"); static storage.  For tests and benchmarks. */
+ * ("warp", "tile", "ring", "rows", "wide", "general", "head", "head_general", "two_pass", "tp", "none"); static storage.  For tests and benchmarks. */
 const char* qknorm_last_variant(void);
 
 /* Number of kernel launches this thread has enqueued through the library. */

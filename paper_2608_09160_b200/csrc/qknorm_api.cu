@@ -588,6 +588,17 @@ int launch(Params& P, cudaStream_t stream) {
         return launch(K, stream);
       }
     }
+    // a tensor beyond 32768 elements: the vectorised two-pass kernel
+    {
+      void (*wide)(const Params) = P.elem_bytes == 1 ? wide_kernel<IoE4m3> : wide_kernel<IoBf16>;
+      int bres = 1;
+      rc = resident_blocks((const void*)wide, kWideThreads, 0, &bres);
+      if (rc != QKNORM_OK) return rc;
+      long long grid = (long long)bres * sms;
+      if (grid > 2 * P.T) grid = 2 * P.T;
+      wide<<<(unsigned)grid, kWideThreads, 0, stream>>>(P);
+      return finish_launch("wide");
+    }
   }
   void (*gen)(const Params) = P.elem_bytes == 1 ? general_kernel<IoE4m3> : general_kernel<IoBf16>;
   int bres = 1;

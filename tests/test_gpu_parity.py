@@ -127,7 +127,7 @@ def test_unaligned_buffers_take_the_general_kernel(libqknorm, skew):
     ("s_prefill_s3", 3, "warp"), ("s_prefill_konly", 2, "warp"), ("s_2305", 4, "warp"),
     ("s_prefill_s16", 16, "warp"), ("s_prefill_s5", 5, "warp"),
     ("s_prefill_wide", 1, "ring"), ("s_prefill_wide", 4, "ring"),
-    ("s_unaligned", 7, "general"), ("s_max", 1, "general"),
+    ("s_unaligned", 7, "general"), ("s_max", 1, "wide"),
 ])
 def test_every_kernel_variant_is_exercised(libqknorm, name, S, variant):
     w = next(x for x in SMALL if x.name == name)
@@ -292,3 +292,11 @@ def test_wide_gqa_rows_in_eight_slices_take_one_launch_per_tensor(libqknorm):
     assert binding.launch_count() == n0 + 2
     assert res["variant"] == "warp"          # of the second (K) launch
     check_against_oracle(w, 8, res)
+
+
+@pytest.mark.parametrize("T,dq,dk,S,in_place", [(300, 49152, 0, 4, True), (700, 65536, 40960, 1, False), (33, 0, 65536, 16, True)])
+def test_tensors_beyond_one_cta_take_the_vectorised_two_pass_kernel(libqknorm, T, dq, dk, S, in_place):
+    w = W.Workload("wide", tokens=T, dq=dq, dk=dk, shards=(S,), seed=323, sigma=2.0)
+    res = run_case(w, S, in_place=in_place)
+    assert res["variant"] == "wide"
+    check_against_oracle(w, S, res)

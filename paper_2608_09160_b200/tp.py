@@ -233,8 +233,8 @@ def clear_status(inbox, stream=None) -> None:
 
 
 class EpochCounter:
-    """Numbers the calls of a group: 1, 2, ...; ``wrapped`` tells the owner that every rank must
-    quiesce and zero its inbox before the number it is about to hand out is used."""
+    """Numbers the calls of a group: 1, 2, ...; ``next_wraps`` tells the owner that the 32-bit number
+    is about to start again at 1, before which every rank must quiesce and zero its inbox."""
 
     def __init__(self, start: int = 0):
         self.last = start
@@ -330,7 +330,13 @@ class Communicator:
                            out_k=(torch.empty_like(k) if out_k is None else out_k) if k is not None else None,
                            inbox=self.inbox, peer_inbox=list(self.peer_inbox), **kw)
 
-    def forward(self, bufs: RankBuffers, eps: float, *, stream=None, wait_limit_us: int = 0) -> int:
+    def prepare(self, bufs: RankBuffers, eps: float) -> PreparedTp:
+        """The call on these buffers with its arguments marshalled once, for a hot loop:
+        ``comm.forward(bufs, eps, prepared=call)`` then only numbers and launches it."""
+        return PreparedTp([bufs], self.N, self.cap, eps)
+
+    def forward(self, bufs: RankBuffers, eps: float, *, stream=None, wait_limit_us: int = 0,
+                prepared: Optional[PreparedTp] = None) -> int:
         ref = bufs.q if bufs.q is not None else bufs.k
         if ref is None or ref.shape[0] == 0:
             return self.epochs.last          # an empty call takes no number
@@ -341,6 +347,8 @@ class Communicator:
         e = self.epochs.next()
         if self.launch is not None:
             self.launch(bufs, self.N, self.cap, eps, e, wait_limit_us)
+        elif prepared is not None:
+            prepared(e, stream, wait_limit_us)
         else:
             qknorm_fwd_tp([bufs], self.N, self.cap, eps, e, wait_limit_us=wait_limit_us, stream=stream)
         return e

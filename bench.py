@@ -28,6 +28,7 @@ implementation of the paper to run): rank 0 only, each step a bounded sample.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -665,6 +666,8 @@ def main():
     ap.add_argument("--tokens", type=int, default=0, help="override the token count (for profiling a small case)")
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "e4m3"], help="storage format of the activations")
     ap.add_argument("--head-dim", type=int, default=0, help="headwise granularity with this head size (needs --shards 1)")
+    ap.add_argument("--one-rank-slice", type=int, default=0,
+                    help="time the column slice one of N tensor-parallel ranks holds, as unsharded rows (short rows)")
     ap.add_argument("--no-table", action="store_true", help="skip the per-config table")
     ap.add_argument("--tp-only", action="store_true",
                     help="only the tensor-parallel rows of the table (all ranks on this GPU), as one JSON object; "
@@ -707,6 +710,12 @@ def main():
     if args.tokens:
         w = W.scaled(w, args.tokens)
     S = args.shards or w.shards[0]
+    if args.one_rank_slice:
+        # what ONE of n tensor-parallel ranks holds of the workload (its column slice), as unsharded rows
+        n = args.one_rank_slice
+        w = dataclasses.replace(w, name=f"{w.name}-slice-of-{n}", dq=w.dq // n, dk=w.dk // n, shards=(1,),
+                                note=f"column slice of one of {n} ranks, unsharded")
+        S = 1
     peak, peak_kind = measured_peak()
 
     def barrier():

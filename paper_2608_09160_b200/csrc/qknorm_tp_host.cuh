@@ -24,7 +24,10 @@ int tp_configure(TpParams& P, int elem_bytes, int sm_count, int* warps_out, int*
   // on B200 (8 ranks on one GPU): tiles of 9-12 KB are fastest, 5 KB and 18 KB both cost 15-30 %.
   const int cq = wq * elem_bytes / 16, ck = wk * elem_bytes / 16;
   const int row_bytes = (wq + wk) * elem_bytes;
-  const int tile_bytes_max = env_int("QKNORM_TP_TILE_BYTES", 12000);
+  // (With a single rank, nothing to exchange and bf16 rows, small tiles and more warps win instead:
+  // rows of 640 and 1280 bytes run 7-8 % faster with tiles of at most 3 KB, longer rows the same.
+  // FP8 rows cost more instructions per byte and lose 20-40 % that way.)
+  const int tile_bytes_max = env_int("QKNORM_TP_TILE_BYTES", (N == 1 && elem_bytes == 2) ? 3000 : 12000);
   const int forced_log_g = env_int("QKNORM_TP_LOG_G", -1);
   int log_g = 5;
   for (int lg = 2; lg <= 5; ++lg) {

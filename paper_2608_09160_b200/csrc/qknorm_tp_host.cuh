@@ -27,7 +27,11 @@ int tp_configure(TpParams& P, int elem_bytes, int sm_count, int* warps_out, int*
   // (With a single rank, nothing to exchange and bf16 rows, small tiles and more warps win instead:
   // rows of 640 and 1280 bytes run 7-8 % faster with tiles of at most 3 KB, longer rows the same.
   // FP8 rows cost more instructions per byte and lose 20-40 % that way.)
-  const int tile_bytes_max = env_int("QKNORM_TP_TILE_BYTES", (N == 1 && elem_bytes == 2) ? 3000 : 12000);
+  // Rows shorter than 2304 bytes still want two tokens per tile (1536-byte rows: 148 us with one,
+  // 109 us with two).
+  int tile_bytes_default = 12000;
+  if (N == 1 && elem_bytes == 2) tile_bytes_default = (row_bytes < 2304 && 2 * row_bytes > 3000) ? 2 * row_bytes : 3000;
+  const int tile_bytes_max = env_int("QKNORM_TP_TILE_BYTES", tile_bytes_default);
   const int forced_log_g = env_int("QKNORM_TP_LOG_G", -1);
   int log_g = 5;
   for (int lg = 2; lg <= 5; ++lg) {

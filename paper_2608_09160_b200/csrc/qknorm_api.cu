@@ -77,11 +77,18 @@ WarpKernel warp_kernel_for(int l, bool exact, int elem_bytes) {
 // Set by a ring kernel whose bounded wait ran out (0 = never happened).
 __device__ __align__(8) int g_ring_error[8] = {0, 0, 0, 0, 0, 0, 0, 0};  // word 0 is the error word; 1-2: where it happened
 
+// Token queues of the warp-per-token kernel: two 64-bit words per slot (tokens handed out, warps
+// gone), zero between launches.  A slot belongs to one stream of one device, and kernels of one
+// stream never run at the same time, so no two launches in flight share a slot.
+constexpr int kQueueSlots = 256;
+__device__ __align__(16) unsigned long long g_token_queue[kQueueSlots][2];
+
 // Built-in scratch of qknorm_baseline_two_pass_static: 1 MiB of device memory that every
 // GPU which loads this library holds until the process exits.  In host code this name is
 // only a handle for cudaGetSymbolAddress, never a device address.
 constexpr size_t kStaticScratchFloats = 262144;
 static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
+
 
 namespace {
 
@@ -91,10 +98,15 @@ thread_local long long tl_launches = 0;
 
 struct DeviceInfo {
   bool known = false;
+  int index = 0;
   int sm_count = 0;
   int smem_per_sm = 0;       // bytes
   int smem_per_block = 0;    // opt-in maximum, bytes
   int* ring_error = nullptr; // device address of g_ring_error on this device
+  unsigned long long* token_queue = nullptr;  // device address of g_token_queue on this device
+  // which stream owns which queue slot (slot i belongs to queue_stream[i]); guarded by g_devices_mutex
+  cudaStream_t queue_stream[kQueueSlots];
+  int queue_slots_used = 0;
 };
 constexpr int kMaxDevices = 64;
 DeviceInfo g_devices[kMaxDevices];
@@ -125,9 +137,41 @@ int current_device(const DeviceInfo** out) {
     // the symbol's name is only a host-side handle: ask for its address on this device
     e = cudaGetSymbolAddress((void**)&d.ring_error, g_ring_error);
     if (e != cudaSuccess) return set_cuda_error(e);
+    e = cudaGetSymbolAddress((void**)&d.token_queue, g_token_queue);
+    if (e != cudaSuccess) return set_cuda_error(e);
+    d.index = dev;
     d.known = true;
   }
   *out = &d;
+  return QKNORM_OK;
+}
+
+// The token queue a launch on `stream` may use, or nullptr when it has to keep the fixed schedule:
+//  * a launch that is being captured into a CUDA graph (the graph can later be replayed on any
+//    stream, next to anything), and the per-thread default stream handle (one handle, a different
+//    stream in every host thread) get no queue;
+//  * every other stream of a device gets a slot of its own the first time it is seen and keeps it
+//    (a destroyed stream's handle may come back as a new stream: still one stream at a time);
+//  * when all slots are taken, further streams get none.
+// The legacy default stream has two handles (0 and cudaStreamLegacy); both map to one slot.
+int token_queue_for(int dev_index, cudaStream_t stream, unsigned long long** out) {
+  *out = nullptr;
+  if (stream == cudaStreamPerThread) return QKNORM_OK;
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  cudaError_t e = cudaStreamIsCapturing(stream, &cap);
+  if (e != cudaSuccess) return set_cuda_error(e);
+  if (cap != cudaStreamCaptureStatusNone) return QKNORM_OK;
+  if (stream == cudaStreamLegacy) stream = nullptr;
+  std::lock_guard<std::mutex> lock(g_devices_mutex);
+  DeviceInfo& d = g_devices[dev_index];
+  int slot = -1;
+  for (int i = 0; i < d.queue_slots_used; ++i)
+    if (d.queue_stream[i] == stream) { slot = i; break; }
+  if (slot < 0 && d.queue_slots_used < kQueueSlots) {
+    slot = d.queue_slots_used++;
+    d.queue_stream[slot] = stream;
+  }
+  if (slot >= 0) *out = d.token_queue + 2 * (size_t)slot;
   return QKNORM_OK;
 }
 
@@ -359,6 +403,30 @@ int finish_launch(const char* variant) {
   return QKNORM_OK;
 }
 
+// Launch with programmatic stream serialisation: the kernel may begin while the previous kernel of
+// the stream is still running; the kernel itself waits for that kernel's completion
+// (griddepcontrol.wait) before its first access to global memory.  QKNORM_PDL=0 (a debug knob)
+// launches the plain way.
+template <class... KArgs, class... Args>
+cudaError_t launch_overlapped(void (*fn)(KArgs...), unsigned grid, unsigned threads, size_t smem, cudaStream_t stream,
+                              Args... args) {
+  if (!env_int("QKNORM_PDL", 1)) {
+    fn<<<grid, threads, smem, stream>>>(args...);
+    return cudaSuccess;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, fn, args...);
+}
+
 #include "qknorm_tp_host.cuh"  // run_tp, launch_tile
 
 // The TMA ring kernel (prefill sizes).  Returns QKNORM_OK with *done = false when
@@ -441,6 +509,12 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   wa.zero_off = wa.k_base + P.S * wa.k_slice_stride;
   wa.stage_bytes = round_up(wa.zero_off + 16, 128);
   wa.error_word = dev.ring_error;
+  wa.queue = nullptr;
+  wa.stagger_cycles = env_int("QKNORM_STAGGER_CYCLES", 900);
+  if (env_int("QKNORM_QUEUE", 1)) {
+    const int qrc = token_queue_for(dev.index, stream, &wa.queue);
+    if (qrc != QKNORM_OK) return qrc;
+  }
   // One row per warp is always in flight.  Measured on B200: throughput peaks when
   // about 76 KB of rows are in flight per SM and falls off slowly beyond that.
   const int in_flight = 76 * 1024;  // holds for both storage formats (FP8 rows are half as long: twice the warps)
@@ -483,7 +557,8 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   const long long needed = (P.T + warps - 1) / warps;
   if (grid > needed) grid = needed;
   int rc = QKNORM_OK;
-  fn<<<(unsigned)grid, warps * 32, smem, stream>>>(P, wa);
+  const cudaError_t e = launch_overlapped(fn, (unsigned)grid, (unsigned)warps * 32u, (size_t)smem, stream, P, wa);
+  if (e != cudaSuccess) return set_cuda_error(e);
   rc = finish_launch("warp");
   *done = rc == QKNORM_OK;
   return rc;
@@ -555,24 +630,8 @@ int launch(Params& P, cudaStream_t stream) {
       long long grid = (long long)bres * sms;  // bounded grid of co-resident CTAs
       if (grid > P.T) grid = P.T;
       apply_plan(P, plan);
-      if (env_int("QKNORM_PDL", 1)) {
-        // allow this launch to begin while the previous kernel of the stream is still running; the
-        // kernel itself waits for that kernel's completion before its first memory access
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)grid);
-        cfg.blockDim = dim3(plan.threads);
-        cfg.dynamicSmemBytes = 0;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        cudaError_t e = cudaLaunchKernelEx(&cfg, fn, P);
-        if (e != cudaSuccess) return set_cuda_error(e);
-      } else {
-        fn<<<(unsigned)grid, plan.threads, 0, stream>>>(P);
-      }
+      const cudaError_t e = launch_overlapped(fn, (unsigned)grid, (unsigned)plan.threads, 0, stream, P);
+      if (e != cudaSuccess) return set_cuda_error(e);
       return finish_launch("rows");
     }
     // Q and K together are too wide for one CTA's registers (more than 32768 elements): the two

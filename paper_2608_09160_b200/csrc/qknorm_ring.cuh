@@ -19,7 +19,8 @@
 // other row is ever written by this CTA.
 //
 // Every wait on an mbarrier is bounded (about one second); a wait that runs
-// out records an error word and the CTA leaves.
+// out records an error word and the whole CTA leaves together, after one more
+// bounded wait for the copies that are still on their way into its stages.
 #pragma once
 #include "qknorm_rowmap.cuh"
 
@@ -162,17 +163,27 @@ ring_kernel(const __grid_constant__ Params P, const int nst, const int stage_byt
   uint32_t phase = 0;
   for (long long i = 0; i < n_my; ++i, par ^= 1) {
     const long long t = first + i * gridDim.x;
-    if (!ptx::mbar_wait_bounded(bar0 + 8u * st, phase)) {
-      atomicCAS(error_word, 0, 1);  // 1 = a stage never arrived
-      return;  // every thread of the CTA waits on the same barrier and leaves here
-    }
+    const bool arrived = ptx::mbar_wait_bounded(bar0 + 8u * st, phase);
     const uint32_t base = smem0 + (uint32_t)st * (uint32_t)stage_bytes;
     uint4 v[N];
 #pragma unroll
     for (int j = 0; j < N; ++j) v[j] = ptx::lds128(base + soff[j]);
     const float a = lane_group_sum(sumsq_chunks<IoBf16, N>(v), P.log_sub);  // Phase A
     if (m.leader) slots[par][m.slot] = a;
-    __syncthreads();  // slots visible; the stage has been read by everyone
+    // slots visible; the stage has been read by everyone.  The same barrier makes the time-out
+    // decision one for the whole CTA: a thread whose wait ran out has only read a stage that may
+    // be incomplete, nothing has been stored yet, and now everybody leaves together.
+    if (__syncthreads_or(arrived ? 0 : 1)) {
+      if (tid == 0) atomicCAS(error_word, 0, 1);  // 1 = a stage never arrived
+      // Before the CTA retires (and its shared memory can go to another CTA) give every copy that
+      // is still on its way one more bounded wait: stage j holds iteration i + ((j - st) mod nst).
+      if (tid < nst) {
+        const long long i2 = i + ((tid - st + nst) % nst);
+        if (i2 < n_my) ptx::mbar_wait_bounded(bar0 + 8u * tid, (uint32_t)((i2 / nst) & 1));
+      }
+      __syncthreads();
+      return;
+    }
     if (tid < 32 && i + nst < n_my) issue(i + nst, st);
     finish_token<IoBf16, N>(P, m, slots[par], v, gm, t);
     if (++st == nst) { st = 0; phase ^= 1u; }

@@ -39,7 +39,15 @@
 // In-place calls are safe: a row is completely in registers before any of it is
 // overwritten, and the only other row the warp touches is its next one.
 // Every mbarrier wait is bounded (about one second); a wait that runs out records
-// an error word and the warp leaves.
+// an error word and the warp leaves as a whole, after one more bounded wait for the
+// copy that may still be on its way into its stage.
+//
+// Token schedule: a bounded persistent grid (Section III-D).  The first two waves of
+// tokens are dealt round-robin; after that a warp takes its next token from a counter
+// of the launch (one atomic add per token, issued a token ahead), so warps that run
+// slower simply take fewer tokens.  Start-up: the warps of a CTA ask for their first
+// rows a few hundred nanoseconds apart, and the kernel may be launched while the
+// previous kernel of the stream is still running (programmatic dependent launch).
 #pragma once
 #include <type_traits>
 
@@ -49,11 +57,11 @@
 namespace qknorm {
 
 constexpr int kWarpMaxCtaWarps = 4;  // the CTA size is a launch parameter: 1..4 warps
-// Registers are shaped for this many resident CTAs of 4 warps (64 / 128 / 168 / 255 registers
+// Registers are shaped for this many resident CTAs of 4 warps (80 / 128 / 168 / 255 registers
 // per thread).  FP8 rows are instruction-bound and gain from a third CTA at 17..24 slots; bf16
 // rows are faster with the registers than with the extra warps.
 __host__ __device__ constexpr int warp_min_blocks(int l, int elem_bytes) {
-  return l <= 8 ? 8 : (l <= 16 ? 4 : ((l <= 24 && elem_bytes == 1) ? 3 : 2));
+  return l <= 8 ? 6 : (l <= 16 ? 4 : ((l <= 24 && elem_bytes == 1) ? 3 : 2));
 }
 
 struct WarpArgs {
@@ -66,6 +74,11 @@ struct WarpArgs {
   int k_base;           // byte offset of the K part inside a stage
   int zero_off;         // byte offset of the 16 zero bytes
   int* error_word;
+  // Token queue of this launch, or nullptr for the fixed round-robin schedule.  Word 0: tokens
+  // handed out beyond the first wave; word 1: warps that have left.  Both are zero when the
+  // kernel starts and the last warp to leave puts them back to zero.
+  unsigned long long* queue;
+  int stagger_cycles;   // SM clock cycles between the first row requests of consecutive warps of a CTA
 };
 
 // EXACT: every lane has all nq / nk chunk slots (S*g == 32 and the slice rows are
@@ -78,6 +91,10 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   __shared__ uint4 gsm[L * GV][32];
   __shared__ __align__(8) unsigned long long bars[kWarpMaxCtaWarps];
 
+  // Programmatic dependent launch (no-ops without the launch attribute): the next kernel of the
+  // stream may start its own launch now; this one sets up its barriers and addresses and then
+  // waits, so no global memory is touched before everything earlier in the stream is complete.
+  asm volatile("griddepcontrol.launch_dependents;");
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int g = 1 << wa.log_g;
@@ -127,25 +144,51 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   const long long first = (long long)blockIdx.x * cta_warps + warp;
   const long long step = (long long)gridDim.x * cta_warps;
   __syncwarp();  // the warp's mbarrier is initialised (lane 0 did it above)
-  if (first < P.T) arm(first);
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Staggered start: warp w of a CTA asks for its first row w * stagger_cycles after warp 0 does.
+  // If all warps of the grid asked at once, all first rows would arrive together, late (the
+  // requests are served side by side), and nothing would be written until then; spread over
+  // about one token time, the warps start in the rhythm they settle into anyway and the first
+  // stores go out after a third of the time.
+  const long long c_entry = wa.stagger_cycles ? clock64() : 0ll;
+  const long long my_delay = (long long)wa.stagger_cycles * warp;
+  if (my_delay == 0 && first < P.T) arm(first);
 
-  // gamma, once per CTA (the first rows are already on their way): slot j of lane `lane`
-  // holds the GV bf16 vectors that go with the lane's j-th chunk; slots dealt round-robin to the warps
+  // gamma, once per CTA: slot j of lane `lane` holds the GV bf16 vectors that go with the lane's
+  // j-th chunk; slots dealt round-robin to the warps.
   bool gamma_f16 = false;
   {
     const uint4* gq = reinterpret_cast<const uint4*>(P.q.gamma[ss]) + (size_t)l * GV;
     const uint4* gk = reinterpret_cast<const uint4*>(P.k.gamma[ss]) + (size_t)l * GV;
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
     bool fits = true;
-    for (int j = warp; j < L; j += cta_warps) {
+    // B slots per batch: all loads of a batch are issued before the first one is used, so staging
+    // costs one or two memory round trips instead of one per slot
+    constexpr int B = (L <= 8 ? 4 : 10) / GV;  // the small-L kernels are held to 64 registers
+    for (int j0 = warp; j0 < L; j0 += B * cta_warps) {
+      uint4 gv[B][GV];
 #pragma unroll
-      for (int v = 0; v < GV; ++v) {
-        uint4 gv = zero;
-        if (j < nvq) gv = __ldg(gq + (size_t)j * g * GV + v);
-        else if (j >= wa.nq4 && j - wa.nq4 < nvk) gv = __ldg(gk + (size_t)(j - wa.nq4) * g * GV + v);
-        gsm[j * GV + v][lane] = gv;
-        if (IO::kF16Gamma)
-          fits = fits && bf16x2_fits_f16(gv.x) && bf16x2_fits_f16(gv.y) && bf16x2_fits_f16(gv.z) && bf16x2_fits_f16(gv.w);
+      for (int b = 0; b < B; ++b) {
+        const int j = j0 + b * cta_warps;
+#pragma unroll
+        for (int v = 0; v < GV; ++v) {
+          gv[b][v] = zero;
+          if (j < nvq) gv[b][v] = __ldg(gq + (size_t)j * g * GV + v);
+          else if (j >= wa.nq4 && j - wa.nq4 < nvk) gv[b][v] = __ldg(gk + (size_t)(j - wa.nq4) * g * GV + v);
+        }
+      }
+#pragma unroll
+      for (int b = 0; b < B; ++b) {
+        const int j = j0 + b * cta_warps;
+        if (j < L) {
+#pragma unroll
+          for (int v = 0; v < GV; ++v) {
+            gsm[j * GV + v][lane] = gv[b][v];
+            if (IO::kF16Gamma)
+              fits = fits && bf16x2_fits_f16(gv[b][v].x) && bf16x2_fits_f16(gv[b][v].y) && bf16x2_fits_f16(gv[b][v].z) &&
+                     bf16x2_fits_f16(gv[b][v].w);
+          }
+        }
       }
     }
     if (IO::kF16Gamma) {
@@ -168,6 +211,10 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
     }
   }
   __syncthreads();  // the last block-level barrier
+  if (my_delay != 0) {
+    while (clock64() - c_entry < my_delay) __nanosleep(64);
+    if (first < P.T) arm(first);
+  }
 
 
   // ---- loop-invariant per-lane offsets ------------------------------------------------------------
@@ -180,11 +227,30 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   unsigned char* yk = reinterpret_cast<unsigned char*>(P.k.y[ss]) + (size_t)l * 16u;
   const unsigned long long q_row = (unsigned long long)P.q.ldy * IO::kBytes, k_row = (unsigned long long)P.k.ldy * IO::kBytes;
 
+  // Which token a warp takes next.  The first two waves are fixed (warp i takes tokens i and
+  // i + step).  With a queue every further token is handed out by one atomic add on the launch's
+  // counter, so a warp on a slow SM simply takes fewer tokens and all warps finish within a token
+  // or two of each other; without a queue warp i goes on with i + 2*step, i + 3*step, ...
+  // The add for the token after next is issued when the next one is armed and its result is read
+  // a whole token later, so its round trip to L2 never holds the warp up.
+  unsigned long long ticket = 0;
+  auto claim_issue = [&]() {
+    if (wa.queue != nullptr && lane == 0) ticket = atomicAdd(wa.queue, 1ull);
+  };
+  auto claim_result = [&](long long after) -> long long {
+    if (wa.queue == nullptr) return after + step;
+    return 2 * step + (long long)__shfl_sync(0xffffffffu, ticket, 0);
+  };
+  long long t = first, t_next = first + step;
+  if (t_next < P.T) claim_issue();
+
   uint32_t phase = 0;
-  for (long long t = first; t < P.T; t += step) {
-    if (!ptx::mbar_wait_bounded(bar, phase)) {
-      atomicCAS(wa.error_word, 0, 2);  // 2 = a warp's stage never arrived
-      return;
+  bool timed_out = false;
+  while (t < P.T) {
+    // one decision for the whole warp: lanes that saw the phase complete must not go on alone
+    if (__any_sync(0xffffffffu, !ptx::mbar_wait_bounded(bar, phase))) {
+      timed_out = true;
+      break;
     }
     phase ^= 1u;
     // ---- drain the stage into registers --------------------------------------------------------
@@ -246,7 +312,12 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
       totk = __shfl_sync(0xffffffffu, pk, 0);
     }
     // every lane's chunks are in registers and have been used: refill the stage with the next token
-    if (t + step < P.T) arm(t + step);
+    long long t_after = P.T;
+    if (t_next < P.T) {
+      arm(t_next);
+      t_after = claim_result(t_next);    // asked for one token ago
+      if (t_after < P.T) claim_issue();  // the one after that
+    }
 
     const float rq = rstd_of(totq, P.q.inv_d, P.eps);
     const float rk = rstd_of(totk, P.k.inv_d, P.eps);
@@ -282,6 +353,28 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
     };
     if (IO::kF16Gamma && gamma_f16) store_pass(std::true_type{});
     else store_pass(std::false_type{});
+    t = t_next;
+    t_next = t_after;
+  }
+  if (timed_out) {
+    // The row this warp waited for never arrived in time.  Record it, then give the copy one more
+    // bounded wait: the CTA must not retire (and hand its shared memory to another CTA) while a
+    // bulk copy into that memory may still land.
+    if (lane == 0) atomicCAS(wa.error_word, 0, 2);  // 2 = a warp's stage never arrived
+    __any_sync(0xffffffffu, !ptx::mbar_wait_bounded(bar, phase));
+  }
+  if (wa.queue != nullptr) {
+    // leave the queue as this launch found it: the last warp out (of all warps of the grid,
+    // with or without tokens, timed out or not) puts both words back to zero
+    __syncwarp();
+    if (lane == 0) {
+      __threadfence();
+      const unsigned long long gone = atomicAdd(wa.queue + 1, 1ull);
+      if (gone + 1ull == (unsigned long long)step) {
+        atomicExch(wa.queue, 0ull);
+        atomicExch(wa.queue + 1, 0ull);
+      }
+    }
   }
 }
 

@@ -144,6 +144,20 @@ def test_results_are_bitwise_reproducible(libqknorm):
     assert torch.equal(a["rq"], b["rq"]) and torch.equal(a["pq"], b["pq"])
 
 
+@pytest.mark.parametrize("S", [1, 4])
+def test_prefill_kernel_is_bitwise_reproducible_with_its_token_queue(libqknorm, S):
+    """The C3 shape at a prefill size (the warp-per-token kernel at 40 chunk slots per lane).
+    Which warp takes which token is decided at run time by the launch's token queue, but a
+    token's arithmetic does not depend on the warp that does it: two runs give the same bits."""
+    w = W.scaled(W.WORKLOADS["C3"], 4099)
+    a = run_case(w, S)
+    assert binding.last_variant() == "warp"
+    b = run_case(w, S)
+    assert np.array_equal(a["q"], b["q"]) and np.array_equal(a["k"], b["k"])
+    assert torch.equal(a["rq"], b["rq"]) and torch.equal(a["rk"], b["rk"])
+    check_against_oracle(w, S, a)
+
+
 def test_sharded_and_unsharded_agree_within_tolerance(libqknorm):
     w = W.scaled(W.WORKLOADS["C2"], 64)
     a = run_case(w, 1)

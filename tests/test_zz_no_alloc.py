@@ -2,8 +2,9 @@
 device memory (its scratch is an array inside the library image).
 
 It must give what qknorm_baseline_two_pass gives with a caller-owned scratch buffer, on
-every call: the built-in array is shared by all calls and keeps the previous call's
-contents, so the test makes two calls in a row on different data.  The file name makes
+every call, and both must agree with the CPU oracle: the built-in array is shared by all
+calls and keeps the previous call's contents, so the test makes two calls in a row on
+different data (the second problem is smaller, so values of the first stay in the array).  The file name makes
 pytest collect it last; the test needs nothing from the tests before it and also passes
 when it is the only one run in a fresh process.
 """
@@ -11,8 +12,10 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2608_09160_b200 import binding
 from paper_2608_09160_b200 import workloads as W
+from tests import gpu_harness as H
 from tests.util import ordinal_distance
 
 pytestmark = pytest.mark.gpu
@@ -21,6 +24,13 @@ pytestmark = pytest.mark.gpu
 def device_shards(w: W.Workload, S: int):
     inp = W.make_inputs(w)
     return {n: [t.cuda() for t in W.shard_columns(inp[n], S)] for n in ("q", "k", "gamma_q", "gamma_k")}
+
+
+def oracle_bits(w: W.Workload):
+    """The fp64 definition on the same seeded inputs, rounded once to bf16."""
+    inp = W.make_inputs(w)
+    return {n: oracle.rmsnorm(W.bf16_bits(inp[n]), W.bf16_bits(inp["gamma_" + n]), w.eps, nthreads=8)["y"]
+            for n in ("q", "k")}
 
 
 def bits(parts):
@@ -49,6 +59,9 @@ def test_static_scratch_matches_caller_scratch_on_two_calls_in_a_row(libqknorm):
         binding.qknorm_baseline_two_pass_static(d["q"], d["k"], d["gamma_q"], d["gamma_k"], w.eps, got_q, got_k)
         torch.cuda.synchronize()
         assert binding.launch_count() - n0 == 2
+        ref = oracle_bits(w)
+        for name, got in (("q", got_q), ("k", got_k)):
+            H.compare_output(bits(got), ref[name], f"{w.name} {name}: built-in scratch against the oracle")
         for name, got, want in (("q", got_q, want_q), ("k", got_k, want_k)):
             dist = ordinal_distance(bits(got), bits(want))
             assert int(dist.max()) <= 1, f"{w.name} {name}: {int(dist.max())} bf16 steps apart"      # the suite's bar
@@ -64,6 +77,9 @@ def test_static_scratch_in_place_and_size_limit(libqknorm):
     binding.qknorm_baseline_two_pass_static(d["q"], d["k"], d["gamma_q"], d["gamma_k"], w.eps, d["q"], d["k"])
     torch.cuda.synchronize()
     assert np.array_equal(bits(d["q"]), bits(want_q)) and np.array_equal(bits(d["k"]), bits(want_k))
+    ref = oracle_bits(w)
+    H.compare_output(bits(d["q"]), ref["q"], "in place, built-in scratch: q against the oracle")
+    H.compare_output(bits(d["k"]), ref["k"], "in place, built-in scratch: k against the oracle")
     # one token more than the built-in array can serve: refused with its own status, nothing launched
     cap = binding.static_scratch_capacity()
     T = cap // (2 * S) + 1

@@ -51,13 +51,30 @@ NOMINAL_HBM_GBS = 8000.0
 L2_BYTES = 126e6          # B200 L2 capacity
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (read + write) per launch of the dominant kernel measured by ncu
-# (dram__bytes_read.sum + dram__bytes_write.sum); None = not captured.
-# C5/S8: a one-pass capture of the full 65536-token launch (summarised under
-# profiles/): 1 208 027 392 bytes read, 1 150 823 936 written.  Reads equal the algorithmic reads; the writes fall
-# 57 MB short of the algorithmic bytes because the call is in place and the last
-# lines written are still dirty in L2 when the kernel ends.
-NCU_DRAM_TRAFFIC_BYTES = {"C5/S8": 1_208_027_392 + 1_150_823_936}
+# DRAM bytes (read + write) per launch of the dominant kernel, measured by ncu
+# (dram__bytes_read.sum + dram__bytes_write.sum).  The figures live in the profile summaries under
+# profiles/ (a line "traffic_bytes_per_launch = N"), so the number in the JSON line and the capture
+# it came from cannot drift apart; `roofline.traffic_source` names the file.
+TRAFFIC_PROFILES = {
+    ("C5", 8, "bf16"): "profiles/warp_kernel_C5_full_size_dram_traffic.md",
+    ("C3", 1, "bf16"): "profiles/warp_kernel_C3_C4_full_set.md",
+}
+
+
+def ncu_traffic(name: str, S: int, io: str):
+    """(bytes per launch or None, profile file or None) for the workload's dominant kernel."""
+    rel = TRAFFIC_PROFILES.get((name, S, io))
+    if rel is None:
+        return None, None
+    try:
+        with open(os.path.join(ROOT, rel)) as fh:
+            for line in fh:
+                key = f"traffic_bytes_per_launch[{name}/S{S}]"
+                if line.strip().startswith(key):
+                    return int(line.split("=")[1].strip().replace(" ", "").replace("_", "")), rel
+    except OSError:
+        pass
+    return None, None
 
 
 def log(*a):
@@ -350,13 +367,14 @@ def copy_rate_same_bytes(nbytes: int, steps: int = 10) -> float:
     return 4 * n / (statistics.median(ts) * 1e-3) / 1e9
 
 
-def config_table(steps: int, warmup: int, peak: float, skip: str):
+def config_table(steps: int, warmup: int, peak: float, skip: str, scope: str = "all"):
     """us/call, GB/s and roofline fraction of every workload other than the headline one."""
     from paper_2608_09160_b200 import binding
     rows = {}
     todo = [(name, S, "bf16") for name, w in W.WORKLOADS.items() for S in w.shards]
-    # FP8-E4M3 activations (Section IV-C), the prefill workloads at their last shard count
-    todo += [(name, W.WORKLOADS[name].shards[-1], "e4m3") for name in ("C3", "C4", "C5")]
+    if scope == "all":
+        # FP8-E4M3 activations (Section IV-C), the prefill workloads at their last shard count
+        todo += [(name, W.WORKLOADS[name].shards[-1], "e4m3") for name in ("C3", "C4", "C5")]
     for name, S, io in todo:
         w = W.WORKLOADS[name]
         key = f"{name}/S{S}" + ("" if io == "bf16" else "/e4m3")
@@ -365,8 +383,13 @@ def config_table(steps: int, warmup: int, peak: float, skip: str):
         case = DeviceCase(w, S, io=io)
         ts = time_calls(case.call, max(steps, 10), max(warmup, 3))
         med, mn = statistics.median(ts), min(ts)
+        torch.cuda.synchronize()
+        b2b = time_region(case.call, max(steps, 10)) / max(steps, 10)
         row = {"us_median": round(med * 1e3, 3), "us_min": round(mn * 1e3, 3),
+               "us_back_to_back": round(b2b * 1e3, 3),
                "GBps": round(case.bytes / (med * 1e-3) / 1e9, 1),
+               "GBps_back_to_back": round(case.bytes / (b2b * 1e-3) / 1e9, 1),
+               "frac_measured_peak_back_to_back": round(case.bytes / (b2b * 1e-3) / 1e9 / peak, 4),
                "frac_measured_peak": round(case.bytes / (med * 1e-3) / 1e9 / peak, 4),
                "frac_nominal_8TBps": round(case.bytes / (med * 1e-3) / 1e9 / NOMINAL_HBM_GBS, 4),
                "bytes": case.bytes, "variant": binding.last_variant(),
@@ -380,10 +403,34 @@ def config_table(steps: int, warmup: int, peak: float, skip: str):
         rows[key] = row
         del case
         torch.cuda.empty_cache()
-    rows.update(variant_rows(steps, warmup, peak))
-    rows.update(baseline_rows(steps, warmup, peak))
-    rows.update(tp_rows(steps, warmup, peak))
+    if scope == "all":
+        rows.update(variant_rows(steps, warmup, peak))
+        rows.update(baseline_rows(steps, warmup, peak))
+        rows.update(tp_rows(steps, warmup, peak))
     return rows
+
+
+def per_config_summary(table: dict, headline_key: str, headline_row: dict) -> dict:
+    """The five workloads of the metric at their shard counts, one compact row each (time of an
+    isolated call, time per call back to back, GB/s and fraction of the measured copy rate from the
+    back-to-back time, kernel variant; decode sizes: CUDA-graph replay with the data in L2 and not)."""
+    out = {headline_key: headline_row}
+    for name, w in W.WORKLOADS.items():
+        for S in w.shards:
+            key = f"{name}/S{S}"
+            r = table.get(key)
+            if r is None:
+                continue
+            row = {"us_median": r["us_median"], "us_back_to_back": r["us_back_to_back"], "variant": r["variant"]}
+            if "us_graph_replay" in r:
+                row["us_graph_replay"] = r["us_graph_replay"]
+                row["us_graph_replay_l2_cold"] = r["us_graph_replay_l2_cold"]
+            else:
+                row["GBps"] = r["GBps_back_to_back"]
+                row["frac"] = r["frac_measured_peak_back_to_back"]
+                row["frac_isolated_median"] = r["frac_measured_peak"]
+            out[key] = row
+    return dict(sorted(out.items()))
 
 
 def tp_rows(steps: int, warmup: int, peak: float, tokens: int = 0):
@@ -614,6 +661,113 @@ def config_of(w: W.Workload, S: int, world: int, variant=None, io: str = "bf16",
     return cfg
 
 
+# ---------------------------------------------------------------------------------
+# column-sharded mode: one rank per GPU, Algorithm 1's scalar exchange between the GPUs
+# ---------------------------------------------------------------------------------
+def tp_rank_inputs(w: W.Workload, world: int, rank: int, io: str = "bf16"):
+    """Rank `rank`'s column slice of the workload (every rank draws the same full tensors from the
+    workload's seed and keeps its own slice: what a column-parallel projection leaves on the rank)."""
+    inp = (W.make_inputs if io == "bf16" else W.make_inputs_e4m3)(w)
+    return {n: W.shard_columns(inp[n], world)[rank].contiguous() for n in ("q", "k", "gamma_q", "gamma_k")}
+
+
+def run_tp_parallel(w: W.Workload, world: int, rank: int, dist, steps: int, warmup: int, *, device="cuda",
+                    io: str = "bf16", ipc=None, launch=None, e2e: bool = False):
+    """The timed region of `--parallelism tp`: every rank holds its column slice, the communicator
+    wires the inboxes, and a step is one `comm.forward` (one launch per rank; the ranks' kernels
+    push their partial sums of squares into each other's inboxes).  Returns this rank's record with
+    the job time already the MAX over ranks.  `ipc` / `launch` are the communicator's stand-ins
+    (tests on CPU); with them nothing here touches CUDA."""
+    from paper_2608_09160_b200 import tp
+    on_gpu = device != "cpu"
+    host = tp_rank_inputs(w, world, rank, io)
+    dev = {n: t.to(device) for n, t in host.items()}
+    out_q = dev["q"] if w.in_place else torch.empty_like(dev["q"])
+    out_k = dev["k"] if w.in_place else torch.empty_like(dev["k"])
+    comm = tp.Communicator(w.tokens, ipc=ipc, launch=launch)
+    bufs = comm.buffers(dev["q"], dev["k"], dev["gamma_q"], dev["gamma_k"], out_q=out_q, out_k=out_k)
+    prepared = comm.prepare(bufs, w.eps) if launch is None else None
+
+    def step():
+        comm.forward(bufs, w.eps, prepared=prepared)
+
+    def barrier():
+        dist.barrier()
+        if on_gpu:
+            torch.cuda.synchronize()
+
+    def timed(fn, n):
+        barrier()
+        if on_gpu:
+            ms = time_region(fn, n)
+        else:
+            t0 = time.perf_counter()
+            for _ in range(n):
+                fn()
+            ms = (time.perf_counter() - t0) * 1e3
+        barrier()
+        return max_over_ranks(ms, dist if world > 1 else None, device)
+
+    for _ in range(warmup):
+        step()
+    first_epoch = comm.epochs.last
+    if launch is None:
+        from paper_2608_09160_b200 import binding
+        n0 = binding.launch_count()
+    total_ms = timed(step, steps)
+    rec = {"ms_per_step": total_ms / steps, "epochs": (first_epoch, comm.epochs.last),
+           "launches": (binding.launch_count() - n0) if launch is None else 0,
+           "variant": binding.last_variant() if launch is None else None,
+           "rank_bytes": 2 * w.tokens * (dev["q"].shape[1] + dev["k"].shape[1]) * dev["q"].element_size()
+                         + (dev["q"].shape[1] + dev["k"].shape[1]) * 2,
+           "job_bytes": case_bytes_of(w, io), "e2e": None}
+    if e2e and on_gpu:
+        pin = {n: host[n].pin_memory() for n in ("q", "k")}
+        back = {n: torch.empty_like(pin[n]).pin_memory() for n in ("q", "k")}
+
+        def e2e_step():
+            dev["q"].copy_(pin["q"], non_blocking=True)
+            dev["k"].copy_(pin["k"], non_blocking=True)
+            step()
+            back["q"].copy_(out_q, non_blocking=True)
+            back["k"].copy_(out_k, non_blocking=True)
+        e2e_step()
+        e_ms = timed(e2e_step, steps)
+        nbytes = sum(pin[n].numel() * pin[n].element_size() for n in ("q", "k"))
+        rec["e2e"] = {"ms_per_step": e_ms / steps, "h2d": nbytes, "d2h": nbytes}
+    rec["status"] = comm.status()
+    comm.close()
+    return rec
+
+
+def tp_line(w: W.Workload, world: int, args, rec: dict, peak: float, peak_kind: str, variant, launches: int, clocks):
+    """The contract line of `--parallelism tp` (rank 0 prints it)."""
+    ms = rec["ms_per_step"]
+    value = rec["job_bytes"] / (ms * 1e-3) / 1e9                 # all ranks' bytes over the slowest rank's time
+    per_gpu = rec["rank_bytes"] / (ms * 1e-3) / 1e9
+    cfg = config_of(w, world, world, variant, args.dtype)
+    cfg["parallelism"] = f"tensor-parallel x{world}, scalar exchange"
+    cfg["bytes_per_step_per_gpu"] = rec["rank_bytes"]
+    e2e = None
+    if rec["e2e"] is not None:
+        e = rec["e2e"]
+        e2e = {"value": round(rec["job_bytes"] / (e["ms_per_step"] * 1e-3) / 1e9, 3), "unit": UNIT,
+               "h2d_bytes_per_step": e["h2d"], "d2h_bytes_per_step": e["d2h"], "ms_per_step": round(e["ms_per_step"], 3),
+               "how": "per rank: the slice from pinned host memory, one call, the slice back to pinned host memory"}
+    return {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms, 5), "higher_is_better": True,
+        "scaling": "strong", "vs_baseline": None, "dtype": "f32", "storage_dtype": args.dtype, "accum_dtype": "f32",
+        "data": "synthetic", "config": cfg, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": round(per_gpu, 1), "peak": peak, "unit": UNIT,
+                     "frac": round(per_gpu / peak, 4), "traffic": None, "peak_kind": f"{peak_kind} device copy rate (hbm_gbs)",
+                     "per_gpu": True, "kernel_variant": variant,
+                     "exchange_bytes_per_step_per_gpu": 16 * w.tokens * (world - 1),
+                     "all_waits_completed": rec["status"].get("status") == 0},
+        "cpu_baseline": None,
+    }
+
+
 def run_reference(args):
     """--impl reference: the oracle as it stands, on host cores, rank 0 only."""
     rank = int(os.environ.get("RANK", "0"))
@@ -643,8 +797,9 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": round(gbs, 4), "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(total / args.steps * 1e3, 3),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {**config_of(w, S, 1), "sample_tokens_per_step": n},
-        "cpu_baseline": {"value": round(gbs, 4), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "config": config_of(w, S, 1),
+        "cpu_baseline": {"value": round(gbs, 4), "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                         "sample_tokens_per_step": n},
         "e2e": {"value": round(gbs, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -669,9 +824,15 @@ def main():
     ap.add_argument("--one-rank-slice", type=int, default=0,
                     help="time the column slice one of N tensor-parallel ranks holds, as unsharded rows (short rows)")
     ap.add_argument("--no-table", action="store_true", help="skip the per-config table")
+    ap.add_argument("--table-scope", default="all", choices=["all", "configs"],
+                    help="configs: only the five workloads of the metric; all: also the FP8, strided, headwise, "
+                         "short-row, stand-in and tensor-parallel rows")
     ap.add_argument("--tp-only", action="store_true",
                     help="only the tensor-parallel rows of the table (all ranks on this GPU), as one JSON object; "
                          "with --tokens for a small case to profile")
+    ap.add_argument("--parallelism", default="tokens", choices=["tokens", "tp"],
+                    help="tokens: every GPU normalises its own token range, no exchange (default); "
+                         "tp: every GPU holds a column slice and the GPUs exchange Algorithm 1's scalars")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-chunks", type=int, default=32, help="token chunks of the host-to-host pipeline")
     ap.add_argument("--no-cpu", action="store_true")
@@ -709,6 +870,25 @@ def main():
     w = W.WORKLOADS[args.workload]
     if args.tokens:
         w = W.scaled(w, args.tokens)
+    if args.parallelism == "tp":
+        own_group = dist is None
+        if own_group:     # one rank: the communicator still wants a process group for its host-side exchange
+            import socket
+            import torch.distributed as dist
+            with socket.socket() as sock:
+                sock.bind(("127.0.0.1", 0))
+                port = sock.getsockname()[1]
+            dist.init_process_group("gloo", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1)
+        peak, peak_kind = measured_peak()
+        sampler = ClockSampler(local)
+        sampler.start()
+        rec = run_tp_parallel(w, world, rank, dist, args.steps, args.warmup, io=args.dtype, e2e=not args.no_e2e)
+        clocks = sampler.stop()
+        if rank == 0:
+            print(json.dumps(tp_line(w, world, args, rec, peak, peak_kind, rec["variant"], rec["launches"], clocks)),
+                  flush=True)
+        dist.destroy_process_group()
+        return 0
     S = args.shards or w.shards[0]
     if args.one_rank_slice:
         # what ONE of n tensor-parallel ranks holds of the workload (its column slice), as unsharded rows
@@ -738,10 +918,12 @@ def main():
     total_ms = time_region(case.call, args.steps)            # THE timed region: K steps, back to back
     barrier()
     launches = binding.launch_count() - n0                   # kernels of this library launched inside it
+    variant = binding.last_variant()                         # the kernel the timed launches ran
     total_ms = max_over_ranks(total_ms, dist, "cuda")
     ms_per_step = total_ms / args.steps
     value = job_value(case.bytes, world, ms_per_step)
-    launch_ms = statistics.mean(per_call)
+    # the kernel's average launch duration over the timed region (one launch per step on this GPU)
+    launch_ms = total_ms / max(launches, 1)
     achieved = case.bytes / (launch_ms * 1e-3) / 1e9
 
     # ---- end to end: host buffers in, host buffers out ----------------------------------------
@@ -758,10 +940,10 @@ def main():
         e2e = {"value": round(job_value(case.bytes, world, e_ms / args.steps), 3), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "ms_per_step": round(e_ms / args.steps, 3), "calls_per_step": e2e_chunks,
+               "kernel_variant": binding.last_variant(),
                "how": "pinned host buffers -> device -> C-ABI call -> pinned host buffers, in token chunks "
                       "(one copy per chunk and direction) so that both copy directions overlap the kernel"}
     clocks = sampler.stop()      # sampled over the device-resident and the end-to-end timed regions
-    variant = binding.last_variant()
     del case
     torch.cuda.empty_cache()
     case_bytes = case_bytes_of(w, args.dtype)
@@ -775,30 +957,60 @@ def main():
 
     table = None
     if not args.no_table and world == 1:
-        table = config_table(args.steps, args.warmup, peak, skip=f"{w.name}/S{S}")
+        table = config_table(args.steps, args.warmup, peak, skip=f"{w.name}/S{S}", scope=args.table_scope)
     cpu = None
     if not args.no_cpu and world == 1:
         cpu = cpu_baseline(w)
 
+    traffic, traffic_source = (ncu_traffic(w.name, S, args.dtype) if not (args.head_dim or args.tokens or args.one_rank_slice)
+                               else (None, None))
+    isolated_med = statistics.median(per_call)
+    roofline = {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": UNIT,
+                "frac": round(achieved / peak, 4), "traffic": traffic, "traffic_source": traffic_source,
+                "peak_kind": f"{peak_kind} device copy rate (hbm_gbs)",
+                "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4),
+                "algorithmic_bytes_per_launch": case_bytes,
+                "same_size_copy_GBps": round(same_size_copy, 1),
+                "kernel_variant": variant,
+                "how": "achieved = algorithmic bytes per launch / (device time of the timed region / launches in it); "
+                       "launches of one stream overlap their start-up with the previous kernel's tail",
+                "launch_us_mean": round(launch_ms * 1e3, 3),
+                # the same launches timed one by one (an event pair around each, so no overlap between them)
+                "launch_us_isolated_median": round(isolated_med * 1e3, 3),
+                "launch_us_isolated_min": round(min(per_call) * 1e3, 3),
+                "frac_isolated_median": round(case_bytes / (isolated_med * 1e-3) / 1e9 / peak, 4)}
+    if table is not None:
+        roofline["per_config"] = per_config_summary(table, f"{w.name}/S{S}", {
+            "us_median": round(isolated_med * 1e3, 3), "us_back_to_back": round(launch_ms * 1e3, 3),
+            "GBps": round(achieved, 1), "frac": round(achieved / peak, 4), "variant": variant})
+
     line = {
         "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "storage_dtype": args.dtype, "accum_dtype": "f32",
+        "data": "synthetic",
         "config": config_of(w, S, world, variant, args.dtype, args.head_dim),
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": UNIT,
-                     "frac": round(achieved / peak, 4), "traffic": NCU_DRAM_TRAFFIC_BYTES.get(f"{w.name}/S{S}") if (args.dtype == "bf16" and not args.head_dim) else None,
-                     "peak_kind": f"{peak_kind} copy rate (of {peak_kind})",
-                     "frac_of_nominal_8TBps": round(achieved / NOMINAL_HBM_GBS, 4),
-                     "algorithmic_bytes_per_launch": case_bytes,
-                     "same_size_copy_GBps": round(same_size_copy, 1),
-                     "launch_us_mean": round(launch_ms * 1e3, 3), "launch_us_min": round(min(per_call) * 1e3, 3)},
+        "roofline": roofline,
         "cpu_baseline": cpu,
     }
     if table is not None:
-        line["configs"] = table
+        # the full table goes to a file and to stderr; the line on stdout stays short enough to be kept whole
+        # (its roofline.per_config and roofline.widened_rows carry the figures)
+        roofline["widened_rows"] = {k: {kk: r[kk] for kk in ("us_median", "GBps", "frac_measured_peak", "variant",
+                                                             "time_relative_to_fused", "fused_us",
+                                                             "latency_reduction_vs_gather_then_norm_pct",
+                                                             "latency_reduction_vs_two_pass_pct") if kk in r}
+                                    for k, r in table.items() if k not in roofline["per_config"]}
+        try:
+            os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
+            with open(os.path.join(ROOT, "gpurun_out", "bench_configs.json"), "w") as fh:
+                json.dump(table, fh, indent=1)
+        except OSError:
+            pass
+        log("configs: " + json.dumps(table))
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

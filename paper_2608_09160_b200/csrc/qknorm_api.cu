@@ -511,7 +511,7 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   wa.error_word = dev.ring_error;
   wa.queue = nullptr;
   wa.stagger_cycles = env_int("QKNORM_STAGGER_CYCLES", 900);
-  if (env_int("QKNORM_QUEUE", 1)) {
+  {
     const int qrc = token_queue_for(dev.index, stream, &wa.queue);
     if (qrc != QKNORM_OK) return qrc;
   }
@@ -552,7 +552,27 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
     }
   }
   if (warps == 0) return QKNORM_OK;  // not even one stage fits: another variant takes the call
-  const int smem = warps * wa.stage_bytes;
+  // The token queue pays where a warp runs at the speed of its own memory round trips (measured on
+  // bf16 rows of 8-20 KB with 4-8 warps per SM, and on FP8 rows with 4: 2-7 % faster).  FP8 rows with
+  // eight or more warps per SM are bound by the SM's instruction issue; there the warps stay level by
+  // themselves and the fixed schedule is 6-9 % faster, so those launches take no queue.
+  const int want_queue = env_int("QKNORM_QUEUE", -1);
+  if (want_queue == 0 || (want_queue < 0 && P.elem_bytes == 1 && ctas_per_sm * warps >= 8)) wa.queue = nullptr;
+  // Shared memory per CTA: what the stages need, raised to the SM's share for `ctas_per_sm` CTAs, so
+  // that one more CTA never fits.  An overlapped launch (the next call of the stream) then gets its
+  // CTAs onto an SM only as this launch's CTAs leave it, exactly `ctas_per_sm` per SM; if an SM could
+  // take more, the early leavers' SMs would fill up twice and others would stay empty.
+  int smem = warps * wa.stage_bytes;
+  {
+    int share = dev.smem_per_sm / ctas_per_sm - 1024 - static_smem;  // 1 KB per CTA is the system's
+    if (share > dev.smem_per_block - static_smem) share = dev.smem_per_block - static_smem;
+    share &= ~127;
+    if (share > smem && env_int("QKNORM_FILL_SMEM", 1)) {
+      smem = share;
+      const int rc2 = allow_dynamic_smem((const void*)fn, smem);
+      if (rc2 != QKNORM_OK) return rc2;
+    }
+  }
   long long grid = (long long)ctas_per_sm * dev.sm_count;  // bounded grid of co-resident CTAs
   const long long needed = (P.T + warps - 1) / warps;
   if (grid > needed) grid = needed;

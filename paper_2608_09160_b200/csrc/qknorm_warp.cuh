@@ -94,6 +94,8 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   // Programmatic dependent launch (no-ops without the launch attribute): the next kernel of the
   // stream may start its own launch now; this one sets up its barriers and addresses and then
   // waits, so no global memory is touched before everything earlier in the stream is complete.
+  // (The host sizes this kernel's shared memory so that no SM can take more CTAs than the grid
+  // gives it: a CTA of the next launch finds room only where a CTA of this one has left.)
   asm volatile("griddepcontrol.launch_dependents;");
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
@@ -227,22 +229,20 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   unsigned char* yk = reinterpret_cast<unsigned char*>(P.k.y[ss]) + (size_t)l * 16u;
   const unsigned long long q_row = (unsigned long long)P.q.ldy * IO::kBytes, k_row = (unsigned long long)P.k.ldy * IO::kBytes;
 
-  // Which token a warp takes next.  The first two waves are fixed (warp i takes tokens i and
-  // i + step).  With a queue every further token is handed out by one atomic add on the launch's
-  // counter, so a warp on a slow SM simply takes fewer tokens and all warps finish within a token
-  // or two of each other; without a queue warp i goes on with i + 2*step, i + 3*step, ...
-  // The add for the token after next is issued when the next one is armed and its result is read
-  // a whole token later, so its round trip to L2 never holds the warp up.
+  // Which token a warp takes next.  Without a queue warp i takes tokens i, i + step, i + 2*step, ...
+  // With a queue only the first two waves are fixed and every further token comes from the launch's
+  // counter, one atomic add per token, so a warp on a slow SM simply takes fewer tokens and all warps
+  // finish within a token or two of each other.  The add for the token after next is issued when the
+  // next one is armed and its result is read a whole token later, so its round trip to L2 (about a
+  // microsecond under load) never holds the warp up.
   unsigned long long ticket = 0;
+  const bool queued = wa.queue != nullptr;
   auto claim_issue = [&]() {
-    if (wa.queue != nullptr && lane == 0) ticket = atomicAdd(wa.queue, 1ull);
+    if (lane == 0) ticket = atomicAdd(wa.queue, 1ull);
   };
-  auto claim_result = [&](long long after) -> long long {
-    if (wa.queue == nullptr) return after + step;
-    return 2 * step + (long long)__shfl_sync(0xffffffffu, ticket, 0);
-  };
+  auto claim_result = [&]() -> long long { return 2 * step + (long long)__shfl_sync(0xffffffffu, ticket, 0); };
   long long t = first, t_next = first + step;
-  if (t_next < P.T) claim_issue();
+  if (queued && t_next < P.T) claim_issue();
 
   uint32_t phase = 0;
   bool timed_out = false;
@@ -315,8 +315,12 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
     long long t_after = P.T;
     if (t_next < P.T) {
       arm(t_next);
-      t_after = claim_result(t_next);    // asked for one token ago
-      if (t_after < P.T) claim_issue();  // the one after that
+      if (!queued) {
+        t_after = t_next + step;
+      } else {
+        t_after = claim_result();          // asked for one token ago
+        if (t_after < P.T) claim_issue();  // the one after that
+      }
     }
 
     const float rq = rstd_of(totq, P.q.inv_d, P.eps);

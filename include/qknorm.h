@@ -144,8 +144,8 @@ int qknorm_fwd_strided_e4m3(const void* q, const void* k, const void* gamma_q, c
                             void* out_q, void* out_k, int64_t ld_out_q, int64_t ld_out_k, void* stream);
 
 /*
- * qknorm_fwd_headwise -- the other granularity Section II-A names: "headwise QK-Norm
- * computes an independent factor for each attention head".  Row t of q is cut into
+ * qknorm_fwd_headwise -- the other granularity Section II-A names, headwise: every
+ * attention head gets a normalisation factor of its own.  Row t of q is cut into
  * dq/head_dim heads of head_dim consecutive columns; every head is normalised on its
  * own, y = x / sqrt(mean over the head of x^2 + eps) * gamma, with the gamma entries of
  * its columns (gamma_q has dq entries; tile a [head_dim] weight if the model shares
@@ -163,8 +163,8 @@ int qknorm_fwd_headwise(const void* q, const void* k, const void* gamma_q, const
                         int64_t ld_out_q, int64_t ld_out_k, float* rstd_q, float* rstd_k, void* stream);
 
 /*
- * FP8-E4M3 activations (Section IV-C: "SwiftQK accumulates local squared sums and
- * cross-GPU scalar reductions in FP32, even for BF16 and FP8-E4M3 activations").
+ * FP8-E4M3 activations (Section IV-C: the local sums of squares and the reduction of the
+ * scalars across shards stay in fp32 whatever format the activations are stored in).
  * The same operation with q, k and the outputs stored as FP8 E4M3 (one byte per
  * element: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities,
  * S.1111.111 = NaN, largest finite value 448).  gamma stays bf16; all arithmetic is

@@ -311,7 +311,7 @@ int qko_rmsnorm_sharded_e4m3(const uint8_t* const* x_shards, const uint16_t* con
 
 /* ---- headwise granularity (Section II-A) ------------------------------------------------------
  *
- * "Headwise QK-Norm computes an independent factor for each attention head": the row is cut
+ * Headwise granularity gives every attention head a factor of its own: the row is cut
  * into H/head_dim heads of head_dim consecutive elements and Eq. 1 is applied to every head on
  * its own (mean over head_dim), with the gamma entries of those columns.  Heads never straddle
  * a tensor-parallel shard, so the sharded form is the same computation on every shard buffer.

@@ -1,8 +1,8 @@
 // Device helpers used by every libqknorm kernel: the two storage formats of the
 // activations (bf16 and FP8-E4M3) as traits, streaming 128-bit loads/stores.
 //
-// All arithmetic is fp32 (Section IV-C: FP32 accumulation "even for BF16 and
-// FP8-E4M3 activations").  Widening is exact for both formats; the result
+// All arithmetic is fp32 (Section IV-C: sums of squares are accumulated in fp32 for
+// both storage formats).  Widening is exact for both formats; the result
 // (x * gamma) * RMS^-1 is rounded ONCE to the storage format, to nearest even
 // (FP8: saturating at +-448).  gamma is bf16 for both.
 #pragma once

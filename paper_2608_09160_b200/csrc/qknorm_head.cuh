@@ -1,4 +1,4 @@
-// Headwise QK-Norm (Section II-A: "an independent factor for each attention head").
+// Headwise QK-Norm (Section II-A: every attention head has a normalisation factor of its own).
 //
 // Every head (head_dim consecutive columns of a row) is normalised on its own:
 // mean over head_dim, the gamma entries of those columns.  Heads are small

@@ -150,17 +150,38 @@ int qknorm_fwd_strided_e4m3(const void* q, const void* k, const void* gamma_q, c
  * own, y = x / sqrt(mean over the head of x^2 + eps) * gamma, with the gamma entries of
  * its columns (gamma_q has dq entries; tile a [head_dim] weight if the model shares
  * it between heads).  Likewise k.  A head never straddles a tensor-parallel shard, so
- * nothing is combined across shards: call this once per shard buffer.
+ * nothing is combined across shards.
  *   ld_*            row strides in elements as in qknorm_fwd_strided (0 = contiguous)
  *   rstd_q, rstd_k  optional [tokens, dq/head_dim] / [tokens, dk/head_dim] fp32, device
- * bf16.  head_dim < 1 or not dividing a width is QKNORM_ERR_HEADS.  Vectorised for
- * head_dim a multiple of 8 up to 256 with 16-byte aligned pointers and strides; any
+ * head_dim < 1 or not dividing a (shard) width is QKNORM_ERR_HEADS.  Vectorised for heads
+ * of a multiple of 16 bytes up to 512 bytes with 16-byte aligned pointers and strides; any
  * other head_dim or alignment takes a general kernel.
+ *   qknorm_fwd_headwise                bf16 rows, optional strides
+ *   qknorm_fwd_headwise_e4m3           the same with q, k and the outputs as FP8-E4M3 (gamma bf16)
+ *   qknorm_fwd_headwise_sharded        the tensors as num_shards column slices (host arrays of
+ *                                      device pointers as in qknorm_fwd_sharded, contiguous rows):
+ *                                      all slices in ONE launch; dq, dk are the FULL widths;
+ *                                      rstd column s * (heads per slice) + h is head h of slice s
+ *   qknorm_fwd_headwise_sharded_e4m3   the same for FP8-E4M3
  */
 int qknorm_fwd_headwise(const void* q, const void* k, const void* gamma_q, const void* gamma_k,
                         int64_t tokens, int32_t dq, int32_t dk, int32_t head_dim,
                         int64_t ld_q, int64_t ld_k, float eps, void* out_q, void* out_k,
                         int64_t ld_out_q, int64_t ld_out_k, float* rstd_q, float* rstd_k, void* stream);
+int qknorm_fwd_headwise_e4m3(const void* q, const void* k, const void* gamma_q, const void* gamma_k,
+                             int64_t tokens, int32_t dq, int32_t dk, int32_t head_dim,
+                             int64_t ld_q, int64_t ld_k, float eps, void* out_q, void* out_k,
+                             int64_t ld_out_q, int64_t ld_out_k, float* rstd_q, float* rstd_k, void* stream);
+int qknorm_fwd_headwise_sharded(const void* const* q_shards, const void* const* k_shards,
+                                const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                                int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, int32_t head_dim,
+                                float eps, void* const* out_q_shards, void* const* out_k_shards,
+                                float* rstd_q, float* rstd_k, void* stream);
+int qknorm_fwd_headwise_sharded_e4m3(const void* const* q_shards, const void* const* k_shards,
+                                     const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                                     int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk,
+                                     int32_t head_dim, float eps, void* const* out_q_shards,
+                                     void* const* out_k_shards, float* rstd_q, float* rstd_k, void* stream);
 
 /*
  * FP8-E4M3 activations (Section IV-C: the local sums of squares and the reduction of the

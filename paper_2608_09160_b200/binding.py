@@ -26,6 +26,9 @@ EXPORTS = (
     "qknorm_fwd_strided",
     "qknorm_fwd_strided_e4m3",
     "qknorm_fwd_headwise",
+    "qknorm_fwd_headwise_e4m3",
+    "qknorm_fwd_headwise_sharded",
+    "qknorm_fwd_headwise_sharded_e4m3",
     "qknorm_baseline_gather_then_norm",
     "qknorm_baseline_two_pass",
     "qknorm_baseline_two_pass_static",
@@ -93,6 +96,11 @@ def load() -> ctypes.CDLL:
     lib.qknorm_fwd_headwise.argtypes = [_vp, _vp, _vp, _vp, i64, i32, i32, i32, i64, i64, f32, _vp, _vp, i64, i64,
                                         _vp, _vp, _vp]
     lib.qknorm_fwd_headwise.restype = ctypes.c_int
+    lib.qknorm_fwd_headwise_e4m3.argtypes = lib.qknorm_fwd_headwise.argtypes
+    lib.qknorm_fwd_headwise_e4m3.restype = ctypes.c_int
+    for fn in (lib.qknorm_fwd_headwise_sharded, lib.qknorm_fwd_headwise_sharded_e4m3):
+        fn.argtypes = [_vpp, _vpp, _vpp, _vpp, i32, i64, i32, i32, i32, f32, _vpp, _vpp, _vp, _vp, _vp]
+        fn.restype = ctypes.c_int
     for fn in (lib.qknorm_baseline_gather_then_norm, lib.qknorm_baseline_two_pass):
         fn.argtypes = [_vpp, _vpp, _vpp, _vpp, i32, i64, i32, i32, f32, _vpp, _vpp, _vp, ctypes.c_size_t, _vp]
         fn.restype = ctypes.c_int
@@ -344,36 +352,92 @@ def qknorm_fwd_strided(q, k, gamma_q, gamma_k, eps: float, out_q=None, out_k=Non
 
 def qknorm_fwd_headwise(q, k, gamma_q, gamma_k, head_dim: int, eps: float, out_q=None, out_k=None, *,
                         rstd_q=None, rstd_k=None, stream=None):
-    """qknorm_fwd_headwise: every head of head_dim columns normalised on its own.  q, k are
-    [T, d] bf16 CUDA views with unit column stride (either may be None); out_* default to new
-    contiguous tensors; rstd_* are optional fp32 [T, d/head_dim]."""
+    """qknorm_fwd_headwise / qknorm_fwd_headwise_e4m3 (chosen by the activations' dtype): every head of
+    head_dim columns normalised on its own.  q, k are [T, d] bf16 or float8_e4m3fn CUDA views with unit
+    column stride (either may be None); out_* default to new contiguous tensors; rstd_* are optional
+    fp32 [T, d/head_dim]."""
     lib = load()
     ref = q if q is not None else k
     if ref is None:
         raise QKNormError(QKNORM_ERR_NULL, "q and k are both None")
+    act = torch.float8_e4m3fn if ref.dtype is torch.float8_e4m3fn else torch.bfloat16
+    cfunc = lib.qknorm_fwd_headwise_e4m3 if act is torch.float8_e4m3fn else lib.qknorm_fwd_headwise
     T = ref.shape[0]
     dq = q.shape[1] if q is not None else 0
     dk = k.shape[1] if k is not None else 0
     ld = [0, 0, 0, 0]
     if q is not None:
         out_q = torch.empty((T, dq), dtype=q.dtype, device=q.device) if out_q is None else out_q
-        ld[0], ld[2] = _expect_rows(q, T, dq, "q"), _expect_rows(out_q, T, dq, "out_q")
+        ld[0], ld[2] = _expect_rows(q, T, dq, "q", act), _expect_rows(out_q, T, dq, "out_q", act)
         _expect(gamma_q, (dq,), torch.bfloat16, "gamma_q")
     if k is not None:
         out_k = torch.empty((T, dk), dtype=k.dtype, device=k.device) if out_k is None else out_k
-        ld[1], ld[3] = _expect_rows(k, T, dk, "k"), _expect_rows(out_k, T, dk, "out_k")
+        ld[1], ld[3] = _expect_rows(k, T, dk, "k", act), _expect_rows(out_k, T, dk, "out_k", act)
         _expect(gamma_k, (dk,), torch.bfloat16, "gamma_k")
     hd = int(head_dim)
     if rstd_q is not None:
         _expect(rstd_q, (T, dq // max(hd, 1)), torch.float32, "rstd_q")
     if rstd_k is not None:
         _expect(rstd_k, (T, dk // max(hd, 1)), torch.float32, "rstd_k")
-    _invoke(lib.qknorm_fwd_headwise, [_ptr(q), _ptr(k), _ptr(gamma_q) if q is not None else None,
-                                      _ptr(gamma_k) if k is not None else None, T, dq, dk, hd, ld[0], ld[1],
-                                      float(eps), _ptr(out_q) if q is not None else None,
-                                      _ptr(out_k) if k is not None else None, ld[2], ld[3], _ptr(rstd_q),
-                                      _ptr(rstd_k)], stream, (q, k, gamma_q, gamma_k, out_q, out_k, rstd_q, rstd_k))
+    _invoke(cfunc, [_ptr(q), _ptr(k), _ptr(gamma_q) if q is not None else None,
+                    _ptr(gamma_k) if k is not None else None, T, dq, dk, hd, ld[0], ld[1],
+                    float(eps), _ptr(out_q) if q is not None else None,
+                    _ptr(out_k) if k is not None else None, ld[2], ld[3], _ptr(rstd_q),
+                    _ptr(rstd_k)], stream, (q, k, gamma_q, gamma_k, out_q, out_k, rstd_q, rstd_k))
     return out_q, out_k
+
+
+def qknorm_fwd_headwise_e4m3(q, k, gamma_q, gamma_k, head_dim: int, eps: float, out_q=None, out_k=None, **kw):
+    """qknorm_fwd_headwise_e4m3: as qknorm_fwd_headwise with float8_e4m3fn activations."""
+    for t, what in ((q, "q"), (k, "k")):
+        if t is not None and t.dtype is not torch.float8_e4m3fn:
+            raise QKNormError(QKNORM_ERR_SHAPE, f"{what}: expected torch.float8_e4m3fn")
+    return qknorm_fwd_headwise(q, k, gamma_q, gamma_k, head_dim, eps, out_q, out_k, **kw)
+
+
+def qknorm_fwd_headwise_sharded(q_shards, k_shards, gamma_q_shards, gamma_k_shards, head_dim: int, eps: float,
+                                out_q_shards=None, out_k_shards=None, *, rstd_q=None, rstd_k=None, stream=None):
+    """qknorm_fwd_headwise_sharded / _e4m3 (chosen by the activations' dtype): headwise granularity on
+    S column slices in one launch.  *_shards as in qknorm_fwd_sharded; rstd_* are optional fp32
+    [T, d/head_dim] with the heads in slice order.  Returns (out_q_shards, out_k_shards)."""
+    lib = load()
+    ref = q_shards if q_shards is not None else k_shards
+    if ref is None:
+        raise QKNormError(QKNORM_ERR_NULL, "q_shards and k_shards are both None")
+    S = len(ref)
+    if S < 1:
+        raise QKNormError(QKNORM_ERR_SHARDS, "need at least one shard")
+    act = torch.float8_e4m3fn if ref[0].dtype is torch.float8_e4m3fn else torch.bfloat16
+    cfunc = lib.qknorm_fwd_headwise_sharded_e4m3 if act is torch.float8_e4m3fn else lib.qknorm_fwd_headwise_sharded
+    T = ref[0].shape[0]
+    wq = q_shards[0].shape[1] if q_shards is not None else 0
+    wk = k_shards[0].shape[1] if k_shards is not None else 0
+
+    def side(xs, gs, outs, w, name):
+        if xs is None:
+            return None, None, None
+        if outs is None:
+            outs = [torch.empty_like(x) for x in xs]
+        if len(xs) != S or len(gs) != S or len(outs) != S:
+            raise QKNormError(QKNORM_ERR_SHARDS, f"{name}: every list must hold {S} shards")
+        for s in range(S):
+            _expect(xs[s], (T, w), act, f"{name}_shards[{s}]")
+            _expect(gs[s], (w,), torch.bfloat16, f"gamma_{name}_shards[{s}]")
+            _expect(outs[s], (T, w), act, f"out_{name}_shards[{s}]")
+        return xs, gs, outs
+
+    q_shards, gamma_q_shards, out_q_shards = side(q_shards, gamma_q_shards, out_q_shards, wq, "q")
+    k_shards, gamma_k_shards, out_k_shards = side(k_shards, gamma_k_shards, out_k_shards, wk, "k")
+    hd = int(head_dim)
+    if rstd_q is not None:
+        _expect(rstd_q, (T, wq * S // max(hd, 1)), torch.float32, "rstd_q")
+    if rstd_k is not None:
+        _expect(rstd_k, (T, wk * S // max(hd, 1)), torch.float32, "rstd_k")
+    _invoke(cfunc, [_array(q_shards, S), _array(k_shards, S), _array(gamma_q_shards, S), _array(gamma_k_shards, S),
+                    S, T, wq * S, wk * S, hd, float(eps), _array(out_q_shards, S), _array(out_k_shards, S),
+                    _ptr(rstd_q), _ptr(rstd_k)], stream,
+            (q_shards, k_shards, gamma_q_shards, gamma_k_shards, out_q_shards, out_k_shards, rstd_q, rstd_k))
+    return out_q_shards, out_k_shards
 
 
 def _baseline(entry, q_shards, k_shards, gamma_q_shards, gamma_k_shards, eps, out_q_shards, out_k_shards,

@@ -520,6 +520,11 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   const int in_flight = 76 * 1024;  // holds for both storage formats (FP8 rows are half as long: twice the warps)
   int rule = (in_flight + wa.stage_bytes / 2) / wa.stage_bytes;
   if (rule < 2) rule = 2;
+  // FP8 rows cost twice the instructions per byte and a short call is over before the steady state
+  // counts: with fewer than 16 rounds of tokens, half as many warps again are faster (measured, warps
+  // per SM: C3 as FP8 8 -> 12, 39.5 -> 37.6 us; C4 as FP8 12 -> 16, 46.4 -> 41.9 us; the 55 rounds of
+  // C5 as FP8 stay fastest with 8).
+  if (P.elem_bytes == 1 && (double)P.T < 16.0 * dev.sm_count * rule) rule = rule * 3 / 2;
   if (rule > 16) rule = 16;
   // Among the (CTAs per SM, warps per CTA) pairs near that, prefer one whose last round of
   // tokens is nearly full: with T / (148 * warps) rounds of several microseconds each, a
@@ -840,48 +845,29 @@ int run_two_pass(Params& P, float* scratch, cudaStream_t stream) {
                              (const float*)scratch);
 }
 
-// Headwise granularity: every head of head_dim columns on its own (unsharded rows, optional strides).
-int run_headwise(const void* q, const void* k, const void* gq, const void* gk, int64_t T, int32_t dq, int32_t dk,
-                 int32_t head_dim, const int64_t* ld, float eps, void* oq, void* ok, float* rstd_q, float* rstd_k,
+// Headwise granularity: every head of head_dim columns on its own.  The tensors come as S column
+// slices (S = 1: whole rows, optional strides); a head never straddles a slice, so the slices are
+// independent and one launch serves them all.
+int run_headwise(int elem_bytes, const void* const* q, const void* const* k, const void* const* gq,
+                 const void* const* gk, int32_t S, int64_t T, int32_t dq, int32_t dk, int32_t head_dim,
+                 const int64_t* ld, float eps, void* const* oq, void* const* ok, float* rstd_q, float* rstd_k,
                  void* stream) {
+  if (S < 1 || S > kMaxShards) return QKNORM_ERR_SHARDS;
   if (T < 0 || dq < 0 || dk < 0 || dq > kMaxDim || dk > kMaxDim) return QKNORM_ERR_SHAPE;
-  if (head_dim < 1 || dq % head_dim != 0 || dk % head_dim != 0) return QKNORM_ERR_HEADS;
-  if (!(eps >= 0.0f)) return QKNORM_ERR_EPS;
-  if (T == 0) return QKNORM_OK;
-  if (dq == 0 && dk == 0) return QKNORM_ERR_SHAPE;
-  if (dq > 0 && (!q || !gq || !oq)) return QKNORM_ERR_NULL;
-  if (dk > 0 && (!k || !gk || !ok)) return QKNORM_ERR_NULL;
-  for (int i = 0; i < 4; ++i)
-    if (ld[i] < 0) return QKNORM_ERR_SHAPE;
-  // the alias rules are those of the layerwise call on the same buffers
+  if (dq % S != 0 || dk % S != 0) return QKNORM_ERR_SHAPE;
+  if (head_dim < 1 || (dq / S) % head_dim != 0 || (dk / S) % head_dim != 0) return QKNORM_ERR_HEADS;
+  if (ld)
+    for (int i = 0; i < 4; ++i)
+      if (ld[i] < 0) return QKNORM_ERR_SHAPE;
+  // pointers, widths, strides and the alias rules are those of the layerwise call on the same buffers
   Params P;
-  memset(&P, 0, sizeof(P));
-  P.T = T;
-  P.S = 1;
-  P.elem_bytes = 2;
-  struct Side {
-    TensorArgs* a;
-    const void* x;
-    const void* g;
-    void* y;
-    int d;
-    float* rstd;
-    int64_t ldx, ldy;
-  } sides[2] = {{&P.q, q, gq, oq, dq, rstd_q, ld[0], ld[2]}, {&P.k, k, gk, ok, dk, rstd_k, ld[1], ld[3]}};
-  for (Side& sd : sides) {
-    sd.a->d = sd.a->w = sd.d;
-    sd.a->ldx = sd.ldx ? sd.ldx : sd.d;
-    sd.a->ldy = sd.ldy ? sd.ldy : sd.d;
-    if (sd.d == 0) continue;
-    if (sd.a->ldx < sd.d || sd.a->ldy < sd.d) return QKNORM_ERR_SHAPE;
-    if ((((uintptr_t)sd.x) | ((uintptr_t)sd.g) | ((uintptr_t)sd.y)) & 1u) return QKNORM_ERR_ALIGN;
-    if (((uintptr_t)sd.rstd) & 3u) return QKNORM_ERR_ALIGN;
-    sd.a->x[0] = sd.x;
-    sd.a->gamma[0] = (const uint16_t*)sd.g;
-    sd.a->y[0] = sd.y;
-    sd.a->rstd = sd.rstd;
-  }
-  int rc = check_alias(P, T, dq ? dq / head_dim : 1, dk ? dk / head_dim : 1);
+  bool empty = true;
+  int rc = prepare(P, &empty, elem_bytes, q, k, gq, gk, S, T, dq, dk, eps, oq, ok, nullptr, nullptr, nullptr, nullptr, ld);
+  if (rc != QKNORM_OK || empty) return rc;
+  if ((((uintptr_t)rstd_q) | ((uintptr_t)rstd_k)) & 3u) return QKNORM_ERR_ALIGN;
+  P.q.rstd = dq ? rstd_q : nullptr;
+  P.k.rstd = dk ? rstd_k : nullptr;
+  rc = check_alias(P, T, dq ? dq / head_dim : 1, dk ? dk / head_dim : 1);
   if (rc != QKNORM_OK) return rc;
 
   const DeviceInfo* dev = nullptr;
@@ -896,37 +882,46 @@ int run_headwise(const void* q, const void* k, const void* gq, const void* gk, i
   HeadSide* hs[2] = {&H.q, &H.k};
   const TensorArgs* ts[2] = {&P.q, &P.k};
   for (int i = 0; i < 2; ++i) {
-    hs[i]->x = ts[i]->x[0];
-    hs[i]->gamma = ts[i]->gamma[0];
-    hs[i]->y = ts[i]->y[0];
+    if (ts[i]->d == 0) continue;
+    for (int sidx = 0; sidx < S; ++sidx) {
+      hs[i]->x[sidx] = ts[i]->x[sidx];
+      hs[i]->gamma[sidx] = ts[i]->gamma[sidx];
+      hs[i]->y[sidx] = ts[i]->y[sidx];
+    }
     hs[i]->rstd = ts[i]->rstd;
-    hs[i]->ldx = ts[i]->ldx * 2;
-    hs[i]->ldy = ts[i]->ldy * 2;
-    hs[i]->nh = ts[i]->d / head_dim;
+    hs[i]->ldx = ts[i]->ldx * elem_bytes;
+    hs[i]->ldy = ts[i]->ldy * elem_bytes;
+    hs[i]->nh = ts[i]->w / head_dim;
+    hs[i]->heads = hs[i]->nh * S;
+    hs[i]->inv_nh = 1.0f / (float)hs[i]->nh;
   }
   const char* force = env_str("QKNORM_FORCE_VARIANT");
-  const bool vec = !(force && strcmp(force, "general") == 0) && head_dim % 8 == 0 && head_dim <= 256 && vector_path_ok(P);
+  const int head_bytes = head_dim * elem_bytes;
+  const bool vec = !(force && strcmp(force, "general") == 0) && head_bytes % 16 == 0 && head_bytes <= 512 && vector_path_ok(P);
+  const bool fp8 = elem_bytes == 1;
   if (vec) {
-    H.hc = head_dim / 8;
+    H.hc = head_bytes / 16;
     H.log_lph = 0;
     while ((1 << H.log_lph) < H.hc) ++H.log_lph;
+    void (*fn)(const HeadParams) = fp8 ? head_kernel<4, IoE4m3> : head_kernel<4, IoBf16>;
     int bres = 1;
-    rc = resident_blocks((const void*)head_kernel<4>, kHeadThreads, 0, &bres);
+    rc = resident_blocks((const void*)fn, kHeadThreads, 0, &bres);
     if (rc != QKNORM_OK) return rc;
     long long grid = (long long)bres * dev->sm_count;
     const long long needed = (T + kHeadThreads / 32 - 1) / (kHeadThreads / 32);
     if (grid > needed) grid = needed;
-    head_kernel<4><<<(unsigned)grid, kHeadThreads, 0, (cudaStream_t)stream>>>(H);
+    fn<<<(unsigned)grid, kHeadThreads, 0, (cudaStream_t)stream>>>(H);
     return finish_launch("head");
   }
+  void (*gen)(const HeadParams) = fp8 ? head_general_kernel<IoE4m3> : head_general_kernel<IoBf16>;
   int bres = 1;
-  rc = resident_blocks((const void*)head_general_kernel, kHeadThreads, 0, &bres);
+  rc = resident_blocks((const void*)gen, kHeadThreads, 0, &bres);
   if (rc != QKNORM_OK) return rc;
   long long grid = (long long)bres * dev->sm_count;
-  const long long items = T * (H.q.nh + H.k.nh);
+  const long long items = T * (H.q.heads + H.k.heads);
   const long long needed = (items + kHeadThreads / 32 - 1) / (kHeadThreads / 32);
   if (grid > needed) grid = needed;
-  head_general_kernel<<<(unsigned)grid, kHeadThreads, 0, (cudaStream_t)stream>>>(H);
+  gen<<<(unsigned)grid, kHeadThreads, 0, (cudaStream_t)stream>>>(H);
   return finish_launch("head_general");
 }
 
@@ -1062,8 +1057,35 @@ int qknorm_fwd_headwise(const void* q, const void* k, const void* gamma_q, const
                         void* out_q, void* out_k, int64_t ld_out_q, int64_t ld_out_k, float* rstd_q,
                         float* rstd_k, void* stream) {
   const int64_t ld[4] = {ld_q, ld_k, ld_out_q, ld_out_k};
-  return qknorm::run_headwise(q, k, gamma_q, gamma_k, tokens, dq, dk, head_dim, ld, eps, out_q, out_k, rstd_q,
-                              rstd_k, stream);
+  return qknorm::run_headwise(2, &q, &k, &gamma_q, &gamma_k, 1, tokens, dq, dk, head_dim, ld, eps, &out_q, &out_k,
+                              rstd_q, rstd_k, stream);
+}
+
+int qknorm_fwd_headwise_e4m3(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,
+                             int32_t dq, int32_t dk, int32_t head_dim, int64_t ld_q, int64_t ld_k, float eps,
+                             void* out_q, void* out_k, int64_t ld_out_q, int64_t ld_out_k, float* rstd_q,
+                             float* rstd_k, void* stream) {
+  const int64_t ld[4] = {ld_q, ld_k, ld_out_q, ld_out_k};
+  return qknorm::run_headwise(1, &q, &k, &gamma_q, &gamma_k, 1, tokens, dq, dk, head_dim, ld, eps, &out_q, &out_k,
+                              rstd_q, rstd_k, stream);
+}
+
+int qknorm_fwd_headwise_sharded(const void* const* q_shards, const void* const* k_shards,
+                                const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                                int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, int32_t head_dim,
+                                float eps, void* const* out_q_shards, void* const* out_k_shards, float* rstd_q,
+                                float* rstd_k, void* stream) {
+  return qknorm::run_headwise(2, q_shards, k_shards, gamma_q_shards, gamma_k_shards, num_shards, tokens, dq, dk,
+                              head_dim, nullptr, eps, out_q_shards, out_k_shards, rstd_q, rstd_k, stream);
+}
+
+int qknorm_fwd_headwise_sharded_e4m3(const void* const* q_shards, const void* const* k_shards,
+                                     const void* const* gamma_q_shards, const void* const* gamma_k_shards,
+                                     int32_t num_shards, int64_t tokens, int32_t dq, int32_t dk, int32_t head_dim,
+                                     float eps, void* const* out_q_shards, void* const* out_k_shards,
+                                     float* rstd_q, float* rstd_k, void* stream) {
+  return qknorm::run_headwise(1, q_shards, k_shards, gamma_q_shards, gamma_k_shards, num_shards, tokens, dq, dk,
+                              head_dim, nullptr, eps, out_q_shards, out_k_shards, rstd_q, rstd_k, stream);
 }
 
 int qknorm_fwd_e4m3(const void* q, const void* k, const void* gamma_q, const void* gamma_k, int64_t tokens,

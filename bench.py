@@ -562,6 +562,29 @@ def variant_rows(steps: int, warmup: int, peak: float):
                          "bytes": w.algorithmic_bytes, "variant": binding.last_variant(), "l2": "inputs larger than L2"}
         del buf, q, k
         torch.cuda.empty_cache()
+    # headwise on the C5 shape as 8 column slices in one launch (bf16), and on whole FP8-E4M3 rows
+    w = W.WORKLOADS["C5"]
+    for key, io in ((f"C5/headwise128/S8-one-launch/in-place", "bf16"), ("C5/headwise128/e4m3/in-place", "e4m3")):
+        inp = (W.make_inputs if io == "bf16" else W.make_inputs_e4m3)(w)
+        eb = 2 if io == "bf16" else 1
+        nbytes = 2 * w.tokens * (w.dq + w.dk) * eb + (w.dq + w.dk) * 2
+        if io == "bf16":
+            d = {n: [t.cuda() for t in W.shard_columns(inp[n], 8)] for n in ("q", "k", "gamma_q", "gamma_k")}
+            fn = binding.prepared(binding.qknorm_fwd_headwise_sharded, d["q"], d["k"], d["gamma_q"], d["gamma_k"], 128,
+                                  w.eps, d["q"], d["k"])
+        else:
+            d = {n: inp[n].cuda() for n in ("q", "k", "gamma_q", "gamma_k")}
+            fn = binding.prepared(binding.qknorm_fwd_headwise_e4m3, d["q"], d["k"], d["gamma_q"], d["gamma_k"], 128,
+                                  w.eps, d["q"], d["k"])
+        del inp
+        ts = time_calls(fn, max(steps, 10), max(warmup, 3))
+        med = statistics.median(ts)
+        gbs = nbytes / (med * 1e-3) / 1e9
+        rows[key] = {"us_median": round(med * 1e3, 3), "us_min": round(min(ts) * 1e3, 3), "GBps": round(gbs, 1),
+                     "frac_measured_peak": round(gbs / peak, 4), "frac_nominal_8TBps": round(gbs / NOMINAL_HBM_GBS, 4),
+                     "bytes": nbytes, "variant": binding.last_variant(), "l2": "inputs larger than L2"}
+        del d, fn
+        torch.cuda.empty_cache()
     # short rows: what ONE of 8 tensor-parallel ranks holds of C5 (its column slice), normalised on
     # its own as unsharded rows -- the shape the tiled kernel exists for
     w = W.Workload("C5-slice", tokens=65536, dq=1024, dk=128, shards=(1,), sigma=2.0, seed=4, in_place=True)
@@ -999,7 +1022,8 @@ def main():
     if table is not None:
         # the full table goes to a file and to stderr; the line on stdout stays short enough to be kept whole
         # (its roofline.per_config and roofline.widened_rows carry the figures)
-        roofline["widened_rows"] = {k: {kk: r[kk] for kk in ("us_median", "GBps", "frac_measured_peak", "variant",
+        roofline["widened_rows"] = {k: {kk: r[kk] for kk in ("us_median", "us_back_to_back", "GBps", "frac_measured_peak",
+                                                             "frac_measured_peak_back_to_back", "variant",
                                                              "time_relative_to_fused", "fused_us",
                                                              "latency_reduction_vs_gather_then_norm_pct",
                                                              "latency_reduction_vs_two_pass_pct") if kk in r}

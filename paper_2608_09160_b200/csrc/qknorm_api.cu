@@ -485,10 +485,12 @@ int warp_slots_needed(const Params& P) {
 }
 
 // The warp-per-token kernel (prefill sizes, gathered rows of up to 40 chunks per lane).
-int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* done) {
+int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* done, int tokens_per_warp = 1) {
   *done = false;
+  if (tokens_per_warp > 1 && P.S != 1) return QKNORM_OK;  // tokens side by side only for unsharded rows
+  const int groups = tokens_per_warp > 1 ? tokens_per_warp : P.S;  // lane groups: tokens of a tile, or slices
   int log_g = 5;
-  while ((P.S << log_g) > 32) --log_g;  // g = largest power of two <= 32 / S
+  while ((groups << log_g) > 32) --log_g;  // g = largest power of two <= 32 / groups
   const int g = 1 << log_g;
   const int cq = P.q.d ? P.q.w * P.elem_bytes / 16 : 0, ck = P.k.d ? P.k.w * P.elem_bytes / 16 : 0;
   WarpArgs wa;
@@ -498,15 +500,20 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   wa.nq4 = round_up(wa.nq, 4);
   const int l = warp_round_up_l(wa.nq4 + wa.nk);
   if (l < 0) return QKNORM_OK;
-  const bool exact = (P.S << log_g) == 32 && cq % g == 0 && ck % g == 0 && wa.nq % 4 == 0 && wa.nk % 4 == 0;
+  wa.tokens_per_warp = tokens_per_warp > 1 ? tokens_per_warp : 1;
+  const long long units = (P.T + wa.tokens_per_warp - 1) / wa.tokens_per_warp;  // tokens, or tiles of tokens
+  const bool exact = (groups << log_g) == 32 && cq % g == 0 && ck % g == 0 && wa.nq % 4 == 0 && wa.nk % 4 == 0 &&
+                     P.T % wa.tokens_per_warp == 0;
   WarpKernel fn = warp_kernel_for(l, exact, P.elem_bytes);
   if (!fn) return QKNORM_OK;
   // stage layout: Q slices, K slices (each slice row followed by the bank skew), 16 zero bytes
-  const int skew = (P.S > 1 && g < 8) ? g * 16 : 0;
-  wa.q_slice_stride = cq ? P.q.w * P.elem_bytes + skew : 0;
-  wa.k_slice_stride = ck ? P.k.w * P.elem_bytes + skew : 0;
-  wa.k_base = P.S * wa.q_slice_stride;
-  wa.zero_off = wa.k_base + P.S * wa.k_slice_stride;
+  // rows of consecutive lane groups start g*16 bytes apart modulo 128, so that the groups that read
+  // in the same quarter-warp hit different banks
+  auto skew_for = [&](int row_bytes) { return (groups > 1 && g < 8) ? ((g * 16 - row_bytes % 128) % 128 + 128) % 128 : 0; };
+  wa.q_slice_stride = cq ? P.q.w * P.elem_bytes + skew_for(P.q.w * P.elem_bytes) : 0;
+  wa.k_slice_stride = ck ? P.k.w * P.elem_bytes + skew_for(P.k.w * P.elem_bytes) : 0;
+  wa.k_base = groups * wa.q_slice_stride;
+  wa.zero_off = wa.k_base + groups * wa.k_slice_stride;
   wa.stage_bytes = round_up(wa.zero_off + 16, 128);
   wa.error_word = dev.ring_error;
   wa.queue = nullptr;
@@ -524,7 +531,7 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   // counts: with fewer than 16 rounds of tokens, half as many warps again are faster (measured, warps
   // per SM: C3 as FP8 8 -> 12, 39.5 -> 37.6 us; C4 as FP8 12 -> 16, 46.4 -> 41.9 us; the 55 rounds of
   // C5 as FP8 stay fastest with 8).
-  if (P.elem_bytes == 1 && (double)P.T < 16.0 * dev.sm_count * rule) rule = rule * 3 / 2;
+  if (P.elem_bytes == 1 && (double)units < 16.0 * dev.sm_count * rule) rule = rule * 3 / 2;
   if (rule > 16) rule = 16;
   // Among the (CTAs per SM, warps per CTA) pairs near that, prefer one whose last round of
   // tokens is nearly full: with T / (148 * warps) rounds of several microseconds each, a
@@ -545,7 +552,7 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
     for (int c = 1; c <= resident && c <= 8; ++c) {
       if (force_ctas && c != force_ctas && !(force_ctas > resident && c == resident)) continue;
       const int per_sm = c * w;
-      const double rounds = (double)P.T / ((double)dev.sm_count * per_sm);
+      const double rounds = (double)units / ((double)dev.sm_count * per_sm);
       const double tail = rounds / (double)(long long)(rounds + 0.999999);
       const int away = per_sm > rule ? per_sm - rule : rule - per_sm;
       const double score = tail - 0.5 * away / rule - 0.001 * c;  // measured: 25 % off the rule costs ~10 %
@@ -562,7 +569,10 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
   // eight or more warps per SM are bound by the SM's instruction issue; there the warps stay level by
   // themselves and the fixed schedule is 6-9 % faster, so those launches take no queue.
   const int want_queue = env_int("QKNORM_QUEUE", -1);
-  if (want_queue == 0 || (want_queue < 0 && P.elem_bytes == 1 && ctas_per_sm * warps >= 8)) wa.queue = nullptr;
+  // Tiles of tokens of at most 4 KB gain nothing either (2-6 % slower with the queue).
+  if (want_queue == 0 || (want_queue < 0 && P.elem_bytes == 1 && ctas_per_sm * warps >= 8) ||
+      (want_queue < 0 && wa.tokens_per_warp > 1 && wa.stage_bytes <= 4608))
+    wa.queue = nullptr;
   // Shared memory per CTA: what the stages need, raised to the SM's share for `ctas_per_sm` CTAs, so
   // that one more CTA never fits.  An overlapped launch (the next call of the stream) then gets its
   // CTAs onto an SM only as this launch's CTAs leave it, exactly `ctas_per_sm` per SM; if an SM could
@@ -579,7 +589,7 @@ int launch_warp(Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* don
     }
   }
   long long grid = (long long)ctas_per_sm * dev.sm_count;  // bounded grid of co-resident CTAs
-  const long long needed = (P.T + warps - 1) / warps;
+  const long long needed = (units + warps - 1) / warps;
   if (grid > needed) grid = needed;
   int rc = QKNORM_OK;
   const cudaError_t e = launch_overlapped(fn, (unsigned)grid, (unsigned)warps * 32u, (size_t)smem, stream, P, wa);
@@ -613,6 +623,25 @@ int launch(Params& P, cudaStream_t stream) {
       if (plan_rows(P, /*latency=*/true, &plan)) {
         const long long most = env_int("QKNORM_ROWS_MAX_TOKENS", plan.threads <= 384 ? 2048 : 1280);
         if (P.T <= most) latency = true;
+      }
+    }
+    if (!latency && !force_rows && !force_ring && P.S == 1) {
+      // short unsharded rows: several tokens side by side per warp
+      // Rows of a few KB and less: R consecutive tokens side by side per warp (2, 4 or 8 with a tile
+      // of at most 9.5 KB; 16 for rows under 384 bytes), so that the per-token work of a warp (barrier
+      // wait, copy issue, shuffle tree, rsqrt) is done once per tile.  Measured on 600 MB of rows of
+      // 256-2560 bytes: 6.0-6.5 TB/s, against 5.6-6.0 TB/s for the three-stage tiled kernel and
+      // 1.5-6.4 TB/s with one token per warp.
+      int tpw = 1;
+      const int row_bytes = (P.q.d + P.k.d) * P.elem_bytes;
+      while (tpw < 8 && 2 * tpw * row_bytes <= 9728) tpw *= 2;
+      if (row_bytes < 384) tpw = 16;
+      tpw = env_int("QKNORM_TOKENS_PER_WARP", tpw);
+      if (tpw > 16) tpw = 16;
+      if (tpw > 1 && !force_tile) {
+        bool done = false;
+        rc = launch_warp(P, *dev, stream, &done, tpw);
+        if (rc != QKNORM_OK || done) return rc;
       }
     }
     if (!latency && !force_rows && !force_ring && !force_warp) {

@@ -79,6 +79,10 @@ struct WarpArgs {
   // kernel starts and the last warp to leave puts them back to zero.
   unsigned long long* queue;
   int stagger_cycles;   // SM clock cycles between the first row requests of consecutive warps of a CTA
+  // Short unsharded rows (S == 1): R > 1 tokens side by side per warp.  The lane groups then serve R
+  // consecutive tokens instead of S slices of one token (stage rows = tokens, nothing is combined
+  // across groups), and the kernel walks over tiles of R tokens instead of tokens.
+  int tokens_per_warp;
 };
 
 // EXACT: every lane has all nq / nk chunk slots (S*g == 32 and the slice rows are
@@ -102,8 +106,11 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   const int g = 1 << wa.log_g;
   const int s = lane >> wa.log_g;
   const int l = lane & (g - 1);
-  const bool active = s < P.S;
-  const int ss = active ? s : 0;
+  const int R = wa.tokens_per_warp;            // 1: lane groups are slices; > 1: lane groups are tokens
+  const int groups = R > 1 ? R : P.S;
+  const bool active = s < groups;
+  const int srow = active ? s : 0;             // which row of the stage the lane's group reads
+  const int ss = R > 1 ? 0 : srow;             // which slice's buffers the lane's group uses
   const int cq = (P.q.w * IO::kBytes) >> 4, ck = (P.k.w * IO::kBytes) >> 4;  // 16-byte chunks per slice row
   const int nvq = EXACT ? wa.nq : ((active && l < cq) ? (cq - l + g - 1) / g : 0);
   const int nvk = EXACT ? wa.nk : ((active && l < ck) ? (ck - l + g - 1) / g : 0);
@@ -118,28 +125,35 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
     ptx::fence_proxy_async();
     *reinterpret_cast<uint4*>(stage + wa.zero_off) = make_uint4(0u, 0u, 0u, 0u);
   }
-  // ---- who issues which bulk copy: lane i < S the Q slice row i, lane S+i the K slice row i ----
-  const bool issue_q = lane < P.S;
-  const int is = issue_q ? lane : lane - P.S;
+  // ---- who issues which bulk copy: lane i < groups the Q row i of the stage, lane groups+i the K row i ----
+  const bool issue_q = lane < groups;
+  const int is = issue_q ? lane : lane - groups;
+  const int my_tok = R > 1 ? is : 0;           // token of the tile this lane's copy fetches
   uint32_t my_bytes = 0, my_dst = 0;
   unsigned long long my_pitch = 0;  // bytes between consecutive rows of the source
   const unsigned char* my_src = nullptr;
-  if (lane < 2 * P.S) {
+  if (lane < 2 * groups) {
     const TensorArgs& A = issue_q ? P.q : P.k;
     if (A.d != 0) {
       my_bytes = (uint32_t)A.w * IO::kBytes;
       my_pitch = (unsigned long long)A.ldx * IO::kBytes;
-      my_src = reinterpret_cast<const unsigned char*>(A.x[is]);
+      my_src = reinterpret_cast<const unsigned char*>(A.x[R > 1 ? 0 : is]);
       my_dst = issue_q ? (uint32_t)is * (uint32_t)wa.q_slice_stride
                        : (uint32_t)wa.k_base + (uint32_t)is * (uint32_t)wa.k_slice_stride;
     }
   }
   const uint32_t row_bytes = ((uint32_t)P.q.d + (uint32_t)P.k.d) * IO::kBytes;
   const uint64_t policy = ptx::policy_evict_first();
-  auto arm = [&](long long t) {  // whole warp
-    if (lane == 0) ptx::mbar_arrive_expect_tx(bar, row_bytes);
+  const long long units = R > 1 ? (P.T + R - 1) / R : P.T;  // what the warps walk over: tokens, or tiles of R tokens
+  auto arm = [&](long long u) {  // whole warp: unit u into the stage
+    const long long tok = u * R + my_tok;
+    if (lane == 0) {
+      const long long left = P.T - u * R;
+      ptx::mbar_arrive_expect_tx(bar, row_bytes * (uint32_t)(left < R ? left : R));
+    }
     __syncwarp();
-    if (my_bytes) ptx::bulk_load(stage_u32 + my_dst, my_src + (unsigned long long)t * my_pitch, my_bytes, bar, policy);
+    if (my_bytes && tok < P.T)
+      ptx::bulk_load(stage_u32 + my_dst, my_src + (unsigned long long)tok * my_pitch, my_bytes, bar, policy);
   };
 
   const int cta_warps = blockDim.x >> 5;
@@ -154,7 +168,7 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   // stores go out after a third of the time.
   const long long c_entry = wa.stagger_cycles ? clock64() : 0ll;
   const long long my_delay = (long long)wa.stagger_cycles * warp;
-  if (my_delay == 0 && first < P.T) arm(first);
+  if (my_delay == 0 && first < units) arm(first);
 
   // gamma, once per CTA: slot j of lane `lane` holds the GV bf16 vectors that go with the lane's
   // j-th chunk; slots dealt round-robin to the warps.
@@ -215,14 +229,14 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   __syncthreads();  // the last block-level barrier
   if (my_delay != 0) {
     while (clock64() - c_entry < my_delay) __nanosleep(64);
-    if (first < P.T) arm(first);
+    if (first < units) arm(first);
   }
 
 
   // ---- loop-invariant per-lane offsets ------------------------------------------------------------
   // inside a stage: chunk l of the lane's Q slice / K slice
-  const uint32_t sq0 = stage_u32 + (uint32_t)ss * (uint32_t)wa.q_slice_stride + (uint32_t)l * 16u;
-  const uint32_t sk0 = stage_u32 + (uint32_t)wa.k_base + (uint32_t)ss * (uint32_t)wa.k_slice_stride + (uint32_t)l * 16u;
+  const uint32_t sq0 = stage_u32 + (uint32_t)srow * (uint32_t)wa.q_slice_stride + (uint32_t)l * 16u;
+  const uint32_t sk0 = stage_u32 + (uint32_t)wa.k_base + (uint32_t)srow * (uint32_t)wa.k_slice_stride + (uint32_t)l * 16u;
   const uint32_t szero = stage_u32 + (uint32_t)wa.zero_off;
   const uint32_t sstride = (uint32_t)g * 16u;
   unsigned char* yq = reinterpret_cast<unsigned char*>(P.q.y[ss]) + (size_t)l * 16u;
@@ -242,11 +256,11 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
   };
   auto claim_result = [&]() -> long long { return 2 * step + (long long)__shfl_sync(0xffffffffu, ticket, 0); };
   long long t = first, t_next = first + step;
-  if (queued && t_next < P.T) claim_issue();
+  if (queued && t_next < units) claim_issue();
 
   uint32_t phase = 0;
   bool timed_out = false;
-  while (t < P.T) {
+  while (t < units) {
     // one decision for the whole warp: lanes that saw the phase complete must not go on alone
     if (__any_sync(0xffffffffu, !ptx::mbar_wait_bounded(bar, phase))) {
       timed_out = true;
@@ -299,8 +313,10 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
     if (g > 2) { pq += __shfl_xor_sync(0xffffffffu, pq, 2); pk += __shfl_xor_sync(0xffffffffu, pk, 2); }
     if (g > 1) { pq += __shfl_xor_sync(0xffffffffu, pq, 1); pk += __shfl_xor_sync(0xffffffffu, pk, 1); }
     // ---- the slices' scalars in ascending slice order -------------------------------------------------
-    float totq = pq, totk = pk;
-    if (P.S > 1) {
+    float totq = pq, totk = pk;  // (R > 1: every lane group keeps its own token's sums)
+    if (R > 1) {
+      __syncwarp();  // every lane has consumed the stage
+    } else if (P.S > 1) {
       totq = 0.f;
       totk = 0.f;
       for (int s2 = 0; s2 < P.S; ++s2) {
@@ -312,30 +328,32 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
       totk = __shfl_sync(0xffffffffu, pk, 0);
     }
     // every lane's chunks are in registers and have been used: refill the stage with the next token
-    long long t_after = P.T;
-    if (t_next < P.T) {
+    long long t_after = units;
+    if (t_next < units) {
       arm(t_next);
       if (!queued) {
         t_after = t_next + step;
       } else {
         t_after = claim_result();          // asked for one token ago
-        if (t_after < P.T) claim_issue();  // the one after that
+        if (t_after < units) claim_issue();  // the one after that
       }
     }
+    const long long tg = R > 1 ? t * R + s : t;   // the token this lane's group works on
+    const bool live = R > 1 ? (active && tg < P.T) : true;
 
     const float rq = rstd_of(totq, P.q.inv_d, P.eps);
     const float rk = rstd_of(totk, P.k.inv_d, P.eps);
-    if (lane == 0) {
-      if (P.q.rstd != nullptr) P.q.rstd[t] = rq;
-      if (P.k.rstd != nullptr) P.k.rstd[t] = rk;
+    if (R > 1 ? (live && l == 0) : lane == 0) {
+      if (P.q.rstd != nullptr) P.q.rstd[tg] = rq;
+      if (P.k.rstd != nullptr) P.k.rstd[tg] = rk;
     }
-    if (active && l == 0) {
-      if (P.q.partials != nullptr) P.q.partials[(long long)s * P.T + t] = pq;
-      if (P.k.partials != nullptr) P.k.partials[(long long)s * P.T + t] = pk;
+    if (active && l == 0 && live) {
+      if (P.q.partials != nullptr) P.q.partials[(long long)ss * P.T + tg] = pq;
+      if (P.k.partials != nullptr) P.k.partials[(long long)ss * P.T + tg] = pk;
     }
     // ---- Phases B/C: (x * gamma) * RMS^-1, the one write ------------------------------------------------
-    unsigned char* dq_ = yq + (unsigned long long)t * q_row;
-    unsigned char* dk_ = yk + (unsigned long long)t * k_row;
+    unsigned char* dq_ = yq + (unsigned long long)tg * q_row;
+    unsigned char* dk_ = yk + (unsigned long long)tg * k_row;
     auto store_pass = [&](auto f16_gamma) {  // the branch on the gamma format stays outside the slot loops
 #pragma unroll
       for (int jb = 0; jb < L; jb += 4) {
@@ -344,7 +362,7 @@ warp_kernel(const __grid_constant__ Params P, const __grid_constant__ WarpArgs w
         const float r = kpart ? rk : rq;
         const float2 r2 = make_float2(r, r);
         unsigned char* dst = kpart ? dk_ + (size_t)(jb - wa.nq4) * sstride : dq_ + (size_t)jb * sstride;
-        const int nv = kpart ? (EXACT ? wa.nk : nvk) - (jb - wa.nq4) : (EXACT ? wa.nq : nvq) - jb;
+        const int nv = !live ? 0 : (kpart ? (EXACT ? wa.nk : nvk) - (jb - wa.nq4) : (EXACT ? wa.nq : nvq) - jb);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const uint4 ga = gsm[(jb + i) * GV][lane], gb = gsm[(jb + i) * GV + GV - 1][lane];

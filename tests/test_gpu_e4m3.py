@@ -22,7 +22,7 @@ SHAPES = [
     ("e_gqa", 2300, 5120, 1024, (8, 1), ("warp", "warp")),
     ("e_mha", 2100, 5120, 5120, (4,), ("warp",)),
     ("e_odd_width", 650, 1000, 136, (1,), ("general",)),          # not a multiple of 16 elements
-    ("e_ragged", 2177, 1008, 144, (1, 3), ("tile", "warp")),       # multiples of 16, ragged over the lanes
+    ("e_ragged", 2177, 1008, 144, (1, 3), ("warp", "warp")),       # multiples of 16, ragged over the lanes
     ("e_tiny", 3, 16, 16, (1,), ("rows",)),
     ("e_konly", 2100, 0, 2048, (2,), ("warp",)),
 ]
@@ -84,6 +84,18 @@ def test_e4m3_matches_oracle(libqknorm, name, T, dq, dk, S, variant, in_place):
     assert run(w, S, in_place) == variant
 
 
+@pytest.mark.parametrize("name,T,dq,dk", [("e_ragged", 2177, 1008, 144), ("e_short", 3001, 2048, 256), ("e_tiny_rows", 2600, 128, 32)])
+@pytest.mark.parametrize("forced", ["tile", None])
+def test_e4m3_short_unsharded_rows(libqknorm, monkeypatch, name, T, dq, dk, forced):
+    """Short FP8 rows: several tokens side by side per warp (variant "warp"), and the three-stage tiled
+    kernel when it is asked for."""
+    if forced:
+        monkeypatch.setenv("QKNORM_FORCE_VARIANT", forced)
+    w = W.Workload(name, tokens=T, dq=dq, dk=dk, shards=(1,), seed=340 + len(name), sigma=1.5)
+    for in_place in (False, True):
+        assert run(w, 1, in_place) == (forced or "warp")
+
+
 def test_e4m3_saturates_and_propagates_nan(libqknorm):
     T, d = 4, 256
     x = torch.zeros((T, d), dtype=torch.float32)
@@ -133,7 +145,7 @@ def test_full_size_e4m3(libqknorm, name):
         print(f"{name} e4m3 {nm}: all {w.tokens} rows, rate at distance 1 {ones / count:.2e}")
 
 
-@pytest.mark.parametrize("dq,dk,variant", [(2048, 512, "tile"), (8192, 1024, "warp")])
+@pytest.mark.parametrize("dq,dk,variant", [(2048, 512, "warp"), (8192, 1024, "warp")])
 def test_e4m3_gamma_outside_fp16_takes_the_bf16_gamma_path(libqknorm, dq, dk, variant):
     """The prefill kernels keep an fp16 copy of gamma when every value fits fp16; one value that
     does not (2^-20, 1e5) must switch the whole call to the bf16-gamma arithmetic with the same result."""
@@ -153,7 +165,7 @@ def test_e4m3_gamma_outside_fp16_takes_the_bf16_gamma_path(libqknorm, dq, dk, va
     assert (W.e4m3_bits(oq.cpu())[:, 77] & 0x7F == 0x7E).mean() > 0.5     # 1e5 * x saturates
 
 
-@pytest.mark.parametrize("T,dq,dk,pad,variant", [(2200, 4096, 1024, 0, "warp"), (2300, 1024, 256, 16, "tile"),
+@pytest.mark.parametrize("T,dq,dk,pad,variant", [(2200, 4096, 1024, 0, "warp"), (2300, 1024, 256, 16, "warp"),
                                                   (40, 2048, 512, 32, "rows")])
 def test_e4m3_rows_strided_inside_a_fused_qkv_buffer(libqknorm, T, dq, dk, pad, variant):
     """FP8 rows that are column blocks of one fused [T, dq + 2*dk (+ pad)] buffer, normalised in place;

@@ -30,7 +30,7 @@ def fused_qkv(w: W.Workload, pad: int = 0):
     (2100, 5120, 1024, 0, "warp"),      # the fused-projection layout at a prefill size
     (16, 4096, 1024, 0, "rows"),       # decode size
     (2150, 2048, 512, 8, "warp"),       # padded rows
-    (2300, 512, 128, 8, "tile"),        # short rows inside a padded fused buffer: several tokens per warp
+    (2300, 512, 128, 8, "warp"),        # short rows inside a padded fused buffer: several tokens per warp
     (33, 1024, 256, 3, "general"),     # row stride not a multiple of 8 elements
 ])
 def test_strided_in_place_in_a_fused_qkv_buffer(libqknorm, T, dq, dk, pad, variant):

@@ -121,9 +121,9 @@ def test_unaligned_buffers_take_the_general_kernel(libqknorm, skew):
 
 @pytest.mark.parametrize("name,S,variant", [
     ("s_t1", 1, "rows"), ("s_149", 8, "rows"), ("s_gqa8", 8, "rows"), ("s_mid_gqa", 1, "rows"), ("s_mid_mha", 2, "rows"),          # few tokens: register-resident rows
-    ("s_prefill_gqa", 8, "warp"), ("s_prefill_gqa", 1, "warp"), ("s_prefill_odd", 1, "tile"),
-    ("s_2305", 1, "tile"), ("s_tile_gqa", 1, "tile"), ("s_tile_tiny", 1, "tile"), ("s_tile_konly", 1, "tile"),
-    ("s_tile_qonly", 1, "tile"),                                               # short unsharded rows: several tokens per warp
+    ("s_prefill_gqa", 8, "warp"), ("s_prefill_gqa", 1, "warp"), ("s_prefill_odd", 1, "warp"),
+    ("s_2305", 1, "warp"), ("s_tile_gqa", 1, "warp"), ("s_tile_tiny", 1, "warp"), ("s_tile_konly", 1, "warp"),
+    ("s_tile_qonly", 1, "warp"),                                               # short unsharded rows: several tokens side by side per warp
     ("s_prefill_s3", 3, "warp"), ("s_prefill_konly", 2, "warp"), ("s_2305", 4, "warp"),
     ("s_prefill_s16", 16, "warp"), ("s_prefill_s5", 5, "warp"),
     ("s_prefill_wide", 1, "ring"), ("s_prefill_wide", 4, "ring"),
@@ -134,6 +134,19 @@ def test_every_kernel_variant_is_exercised(libqknorm, name, S, variant):
     res = run_case(w, S)
     assert res["variant"] == variant, (name, S, res["variant"])
     check_against_oracle(w, S, res)
+
+
+@pytest.mark.parametrize("name", ["s_2305", "s_tile_gqa", "s_tile_tiny", "s_tile_konly", "s_tile_qonly", "s_prefill_odd"])
+def test_three_stage_tiled_kernel_on_short_unsharded_rows(libqknorm, monkeypatch, name):
+    """Short unsharded rows normally go to the warp-per-tile form of the prefill kernel; the three-stage
+    tiled kernel (the tensor-parallel kernel with a single rank) still serves them when asked to."""
+    monkeypatch.setenv("QKNORM_FORCE_VARIANT", "tile")
+    w = next(x for x in SMALL if x.name == name)
+    res = run_case(w, 1)
+    assert res["variant"] == "tile"
+    check_against_oracle(w, 1, res)
+    res = run_case(w, 1, in_place=True, stats=False)
+    check_against_oracle(w, 1, res)
 
 
 def test_results_are_bitwise_reproducible(libqknorm):

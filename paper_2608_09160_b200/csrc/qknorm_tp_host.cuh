@@ -225,12 +225,11 @@ int run_tp(int elem_bytes, const qknorm_tp_rank* ranks, int n_local, int N, long
 
 
 
-// Unsharded rows too short for one token per warp (a few KB): the tiled kernel with a single rank
-// and therefore no exchange -- several tokens side by side per warp, three stages per warp.
-// Measured on B200, 600 MB of rows: at 640-byte rows the warp-per-token kernel reaches 1.5 TB/s
-// and this one 5.5 TB/s; they meet near 2.8 KB (bf16) and 4 KB (FP8-E4M3), above which the
-// warp-per-token kernel is 5-8 % faster.  Returns QKNORM_OK with *done = false when the call is
-// not of that kind.
+// Unsharded rows on the tiled kernel with a single rank and therefore no exchange -- several tokens
+// side by side per warp, three stages per warp.  Short rows are normally served by the warp kernel
+// with several tokens per warp (6.0-6.5 TB/s against 5.6-6.0 TB/s here); this path remains for
+// QKNORM_FORCE_VARIANT=tile and for shapes the warp kernel has no instantiation for.  Returns
+// QKNORM_OK with *done = false when the call is not of that kind.
 int launch_tile(const Params& P, const DeviceInfo& dev, cudaStream_t stream, bool* done) {
   *done = false;
   if (P.S != 1) return QKNORM_OK;

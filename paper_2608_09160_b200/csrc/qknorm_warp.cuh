@@ -42,6 +42,13 @@
 // an error word and the warp leaves as a whole, after one more bounded wait for the
 // copy that may still be on its way into its stage.
 //
+// Short unsharded rows (tokens_per_warp = R > 1).  The same kernel with the lane groups
+// serving R consecutive TOKENS instead of S slices of one token: the stage holds a tile
+// of R rows, every group keeps its own sums of squares (nothing is combined across
+// groups), and the warp walks over tiles.  The per-token work of a warp (barrier wait,
+// copy issue, shuffle tree, rsqrt, queue) is then done once per R tokens, which is what
+// rows of a few hundred bytes need.
+//
 // Token schedule: a bounded persistent grid (Section III-D).  The first two waves of
 // tokens are dealt round-robin; after that a warp takes its next token from a counter
 // of the launch (one atomic add per token, issued a token ahead), so warps that run

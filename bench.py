@@ -856,6 +856,7 @@ def main():
     ap.add_argument("--parallelism", default="tokens", choices=["tokens", "tp"],
                     help="tokens: every GPU normalises its own token range, no exchange (default); "
                          "tp: every GPU holds a column slice and the GPUs exchange Algorithm 1's scalars")
+    ap.add_argument("--configs-out", default="", help="also write the full per-config table to this JSON file")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-chunks", type=int, default=32, help="token chunks of the host-to-host pipeline")
     ap.add_argument("--no-cpu", action="store_true")
@@ -1020,7 +1021,7 @@ def main():
         "cpu_baseline": cpu,
     }
     if table is not None:
-        # the full table goes to a file and to stderr; the line on stdout stays short enough to be kept whole
+        # the full table goes to stderr (and to --configs-out); the line on stdout stays short enough to be kept whole
         # (its roofline.per_config and roofline.widened_rows carry the figures)
         roofline["widened_rows"] = {k: {kk: r[kk] for kk in ("us_median", "us_back_to_back", "GBps", "frac_measured_peak",
                                                              "frac_measured_peak_back_to_back", "variant",
@@ -1028,12 +1029,13 @@ def main():
                                                              "latency_reduction_vs_gather_then_norm_pct",
                                                              "latency_reduction_vs_two_pass_pct") if kk in r}
                                     for k, r in table.items() if k not in roofline["per_config"]}
-        try:
-            os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-            with open(os.path.join(ROOT, "gpurun_out", "bench_configs.json"), "w") as fh:
-                json.dump(table, fh, indent=1)
-        except OSError:
-            pass
+        if args.configs_out:
+            try:
+                os.makedirs(os.path.dirname(os.path.abspath(args.configs_out)), exist_ok=True)
+                with open(args.configs_out, "w") as fh:
+                    json.dump(table, fh, indent=1)
+            except OSError as e:
+                log(f"could not write {args.configs_out}: {e}")
         log("configs: " + json.dumps(table))
     print(json.dumps(line), flush=True)
     if dist is not None:

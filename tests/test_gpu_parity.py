@@ -149,6 +149,28 @@ def test_three_stage_tiled_kernel_on_short_unsharded_rows(libqknorm, monkeypatch
     check_against_oracle(w, 1, res)
 
 
+def test_one_slice_through_the_sharded_entry_point_on_short_rows(libqknorm):
+    """S = 1 through qknorm_fwd_sharded_ex on rows short enough for several tokens per warp: the
+    slice's scalar is the row's sum of squares, one per token, whichever lane group served the token."""
+    w = next(x for x in SMALL if x.name == "s_tile_gqa")
+    inp = W.make_inputs(w)
+    T = w.tokens
+    dev = {k: [v.cuda()] for k, v in inp.items()}
+    pq = torch.full((1, T), float("nan"), device="cuda")
+    pk = torch.full((1, T), float("nan"), device="cuda")
+    rq = torch.full((T,), float("nan"), device="cuda")
+    rk = torch.full((T,), float("nan"), device="cuda")
+    oq, ok = binding.qknorm_fwd_sharded(dev["q"], dev["k"], dev["gamma_q"], dev["gamma_k"], w.eps,
+                                        partials_q=pq, partials_k=pk, rstd_q=rq, rstd_k=rk)
+    torch.cuda.synchronize()
+    assert binding.last_variant() == "warp"
+    for nm, out, p, r in (("q", oq, pq, rq), ("k", ok, pk, rk)):
+        sh = oracle.rmsnorm_sharded([W.bf16_bits(inp[nm])], [W.bf16_bits(inp["gamma_" + nm])], w.eps, nthreads=NTHREADS)
+        H.compare_output(H.bits(out[0]), sh["y"][0], f"one slice {nm}")
+        H.compare_stat(p, sh["partials"], f"one slice partials {nm}")
+        H.compare_stat(r, sh["rstd"], f"one slice rstd {nm}")
+
+
 def test_results_are_bitwise_reproducible(libqknorm):
     w = next(x for x in SMALL if x.name == "s_gqa8")
     a = run_case(w, 8)

@@ -21,15 +21,19 @@
  *  - Pointer ARRAYS (the *_shards arguments) are HOST arrays of device pointers.
  *    They are read during the call only and may be freed on return.
  *  - Ownership: the caller owns every buffer.  The library allocates nothing on
- *    the device, frees nothing, and keeps no state except a per-device cache of
- *    the SM count and kernel occupancy.
+ *    the device and frees nothing.  Its own state: a per-device cache of the SM
+ *    count and kernel occupancy on the host, and a few KB of device memory inside
+ *    the library image (an error word; 256 token counters, one per stream that has
+ *    made a prefill-size call, each back at zero when its kernel ends).
  *  - Asynchrony: work is enqueued on `stream` (a cudaStream_t passed as void*;
  *    NULL = the legacy default stream) and the call returns without
  *    synchronising.  No cudaMalloc, no cudaMemcpy, no host synchronisation.
- *    Calls of up to about two thousand tokens are launched with programmatic stream
+ *    Decode-size and prefill-size calls are launched with programmatic stream
  *    serialisation: the launch may begin while the previous kernel of the stream is still
  *    running, and the kernel waits for that kernel to complete (and its writes to be
  *    visible) before its first memory access, so stream order is kept as usual.
+ *    Calls on different streams may run at the same time; calls may be captured into
+ *    CUDA graphs.
  *  - Errors: the return value is a qknorm_status.  On any error nothing has
  *    been launched.  tokens == 0 returns QKNORM_OK without a launch.
  *  - A tensor can be skipped: dq == 0 (with its pointers ignored) means "K
@@ -40,7 +44,9 @@
  *  - Precision: inputs are widened to fp32 (exact), sums of squares and all
  *    arithmetic are fp32, the product x*gamma*rstd is rounded ONCE to bf16
  *    (round to nearest even).  Subnormals are kept.  Results are bitwise
- *    reproducible run to run (no atomics).
+ *    reproducible run to run: prefill-size calls hand tokens to warps through a
+ *    counter, but a token's arithmetic does not depend on the warp that does it,
+ *    and no value is ever accumulated with atomics.
  *  - Fast path: when every base pointer is 16-byte aligned and every (shard)
  *    width is a multiple of 8 elements, vectorised kernels run; any other
  *    width or alignment is served by a slower general kernel, not an error.  A call is

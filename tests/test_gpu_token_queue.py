@@ -125,3 +125,24 @@ def test_captured_prefill_call_replays_next_to_eager_calls(libqknorm):
     check(w, inp, g_oq, g_ok, "graph replay")
     check(w, inp, e_oq, e_ok, "eager next to the replay")
     assert binding.device_error_word() == 0
+
+
+def test_per_thread_default_stream_handle_takes_no_counter(libqknorm):
+    """cudaStreamPerThread is ONE handle value that names a different stream in every host thread, so a
+    counter keyed by it could be shared by kernels that run at the same time: such launches keep the
+    fixed schedule.  The result is the same as on an ordinary stream."""
+    CUDA_STREAM_PER_THREAD = 2
+    w = W.Workload("queue_ptds", tokens=3100, dq=5120, dk=1024, shards=(1,), seed=74)
+    inp = W.make_inputs(w)
+    q, k = inp["q"].cuda(), inp["k"].cuda()
+    gq, gk = inp["gamma_q"].cuda(), inp["gamma_k"].cuda()
+    torch.cuda.synchronize()
+    a_q, a_k = binding.qknorm_fwd(q, k, gq, gk, w.eps)
+    b_q, b_k = torch.empty_like(q), torch.empty_like(k)
+    binding.qknorm_fwd(q, k, gq, gk, w.eps, b_q, b_k, stream=CUDA_STREAM_PER_THREAD)
+    assert binding.last_variant() == "warp"
+    torch.cuda.synchronize()
+    assert torch.equal(a_q, b_q) and torch.equal(a_k, b_k)
+    ref = H.oracle_unsharded(inp, w.eps, nthreads=NTHREADS)
+    H.compare_output(H.bits(b_q), ref["q"]["y"], "per-thread default stream q")
+    H.compare_output(H.bits(b_k), ref["k"]["y"], "per-thread default stream k")
